@@ -1,0 +1,166 @@
+"""Double-precision CPU oracle for the nested Forward-AD activation pass.
+
+TEST INFRASTRUCTURE.  Only the test-suite, the smoke check and the benchmark's
+``cpu_baseline`` / ``--impl reference`` legs may import this package; the CUDA
+library never does, and this package imports nothing of the CUDA library.
+
+The arithmetic lives in ``nfad_oracle.c`` (plain C, fp64, one expression per
+quantity: Table I for the activations, Table II / Eq. 3 for the derivatives,
+Eq. 4 for the backward product).  This module compiles that file with gcc on
+first use and marshals numpy arrays into it.  Stored tensors cross the boundary
+as raw bit patterns: ``float32`` arrays for fp32, ``uint16`` arrays for bf16 and
+fp16.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+import threading
+
+import numpy as np
+
+KINDS = {"gelu_erf": 0, "gelu_tanh": 1, "swish": 2, "mish": 3}
+DTYPES = {"f32": 0, "bf16": 1, "f16": 2}
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "nfad_oracle.c")
+_LIB = os.path.join(_HERE, "libnfad_oracle.so")
+_lock = threading.Lock()
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc (IEEE semantics: no fast-math, no contraction)."""
+    with _lock:
+        stale = (not os.path.exists(_LIB)) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC)
+        if force or stale:
+            cmd = ["gcc", "-O2", "-std=c11", "-fPIC", "-shared", "-fopenmp",
+                   "-ffp-contract=off", "-fno-fast-math", "-o", _LIB, _SRC, "-lm"]
+            subprocess.run(cmd, check=True, capture_output=True)
+    return _LIB
+
+
+class _Point(ctypes.Structure):
+    _fields_ = [("f", ctypes.c_double), ("fprime", ctypes.c_double),
+                ("term_h", ctypes.c_double), ("term_xh", ctypes.c_double)]
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        lib = ctypes.CDLL(build())
+        vp, sz, ci = ctypes.c_void_p, ctypes.c_size_t, ctypes.c_int
+        lib.nfad_oracle_eval_point.argtypes = [ci, ctypes.c_double, ctypes.POINTER(_Point)]
+        lib.nfad_oracle_forward.argtypes = [ci, ci, vp, sz, vp, vp, vp]
+        lib.nfad_oracle_round.argtypes = [ci, vp, sz, vp]
+        lib.nfad_oracle_widen.argtypes = [ci, vp, sz, vp]
+        lib.nfad_oracle_backward.argtypes = [ci, vp, vp, sz, vp]
+        lib.nfad_oracle_forward_backward.argtypes = [ci, ci, vp, vp, sz, vp, vp, vp]
+        lib.nfad_oracle_set_threads.argtypes = [ci]
+        for name in ("nfad_oracle_eval_point", "nfad_oracle_forward", "nfad_oracle_round",
+                     "nfad_oracle_widen", "nfad_oracle_backward", "nfad_oracle_forward_backward",
+                     "nfad_oracle_get_threads", "nfad_oracle_max_threads"):
+            getattr(lib, name).restype = ci
+        lib.nfad_oracle_set_threads.restype = None
+        _lib = lib
+    return _lib
+
+
+def _code(table, key):
+    return table[key] if isinstance(key, str) else int(key)
+
+
+def _storage_np(dtype) -> np.dtype:
+    return np.dtype(np.float32) if _code(DTYPES, dtype) == 0 else np.dtype(np.uint16)
+
+
+def _check_storage(a: np.ndarray, dtype) -> np.ndarray:
+    want = _storage_np(dtype)
+    if a.dtype != want:
+        raise TypeError(f"stored tensor for dtype {dtype!r} must be a {want} array of raw values, got {a.dtype}")
+    return np.ascontiguousarray(a).reshape(-1)
+
+
+def _ptr(a: np.ndarray):
+    return ctypes.c_void_p(a.ctypes.data)
+
+
+def _ok(rc: int, what: str):
+    if rc != 0:
+        raise ValueError(f"{what}: oracle status {rc}")
+
+
+def set_threads(t: int) -> None:
+    _load().nfad_oracle_set_threads(int(t))
+
+
+def get_threads() -> int:
+    return _load().nfad_oracle_get_threads()
+
+
+def max_threads() -> int:
+    """Cores the process may run on (what an all-core timing uses)."""
+    try:
+        return len(os.sched_getaffinity(0))
+    except AttributeError:
+        return _load().nfad_oracle_max_threads()
+
+
+def eval_point(kind, x: float):
+    """(f, f', h, x h') at one double x; f' = h + x h' (product rule, Eq. 3)."""
+    p = _Point()
+    _ok(_load().nfad_oracle_eval_point(_code(KINDS, kind), float(x), ctypes.byref(p)), "eval_point")
+    return p.f, p.fprime, p.term_h, p.term_xh
+
+
+def forward(kind, dtype, x: np.ndarray, want_cond: bool = False):
+    """Unrounded f(x), f'(x) in fp64 for a stored tensor x; optionally |h| + |x h'|."""
+    x = _check_storage(x, dtype)
+    n = x.size
+    f = np.empty(n, np.float64)
+    fp = np.empty(n, np.float64)
+    cond = np.empty(n, np.float64) if want_cond else None
+    _ok(_load().nfad_oracle_forward(_code(KINDS, kind), _code(DTYPES, dtype), _ptr(x), n,
+                                    _ptr(f), _ptr(fp), _ptr(cond) if want_cond else None), "forward")
+    return (f, fp, cond) if want_cond else (f, fp)
+
+
+def round_to(dtype, v: np.ndarray) -> np.ndarray:
+    """One round-to-nearest-even from fp64 to the storage type (raw bit patterns)."""
+    v = np.ascontiguousarray(v, np.float64).reshape(-1)
+    out = np.empty(v.size, _storage_np(dtype))
+    _ok(_load().nfad_oracle_round(_code(DTYPES, dtype), _ptr(v), v.size, _ptr(out)), "round_to")
+    return out
+
+
+def widen(dtype, a: np.ndarray) -> np.ndarray:
+    """Stored values to fp64 (exact)."""
+    a = _check_storage(a, dtype)
+    out = np.empty(a.size, np.float64)
+    _ok(_load().nfad_oracle_widen(_code(DTYPES, dtype), _ptr(a), a.size, _ptr(out)), "widen")
+    return out
+
+
+def backward(dtype, grad_out: np.ndarray, fprime_saved: np.ndarray) -> np.ndarray:
+    """grad_in = RN(grad_out * f'_saved), the product formed exactly in fp64 (Eq. 4)."""
+    g = _check_storage(grad_out, dtype)
+    d = _check_storage(fprime_saved, dtype)
+    if g.size != d.size:
+        raise ValueError("size mismatch")
+    out = np.empty(g.size, _storage_np(dtype))
+    _ok(_load().nfad_oracle_backward(_code(DTYPES, dtype), _ptr(g), _ptr(d), g.size, _ptr(out)), "backward")
+    return out
+
+
+def forward_backward(kind, dtype, x: np.ndarray, grad_out: np.ndarray):
+    """The whole path on the CPU: (y, f'_saved, grad_in) as stored tensors. Used for timing."""
+    x = _check_storage(x, dtype)
+    g = _check_storage(grad_out, dtype)
+    if g.size != x.size:
+        raise ValueError("size mismatch")
+    st = _storage_np(dtype)
+    y, d, gin = (np.empty(x.size, st) for _ in range(3))
+    _ok(_load().nfad_oracle_forward_backward(_code(KINDS, kind), _code(DTYPES, dtype), _ptr(x), _ptr(g),
+                                             x.size, _ptr(y), _ptr(d), _ptr(gin)), "forward_backward")
+    return y, d, gin
