@@ -1,0 +1,384 @@
+#!/usr/bin/env python
+"""Benchmark of the nested Forward-AD activation pass on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
+
+One step = one pass of the whole hot path over one batch of the workload: for
+every activation kind the workload names, forward (x -> y, f') and backward
+(g, f' -> grad_in), each one kernel launched through the C-ABI binding.  The
+default workload is the BERT-base feed-forward activation (bf16 [32,128,3072],
+GELU erf and tanh forms).  Prints ONE JSON line.
+
+Timing: CUDA events on the launching stream; W >= 3 warm-up steps; buffer sets
+are rotated so that the bytes touched between two uses of a buffer exceed 4x the
+L2 capacity, and backward consumes the f' that a forward wrote half a rotation
+earlier (as in training, where backward comes long after forward), so no tensor
+is served from L2.  With N > 1 every rank runs the same workload on its own GPU
+(the path has no exchange step: weak scaling, no collective in the data path);
+the barrier and the max-over-ranks of the device time use torch.distributed.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "fwd+bwd elements/s"
+UNIT = "elements/s"
+L2_BYTES = 126 * 1024 * 1024
+FALLBACK_HBM_GBS = 6650.0          # an earlier copy-bandwidth measurement on this machine's B200s
+
+# DRAM bytes per element (read + write) of the dominant kernel measured by ncu
+# (dram__bytes_read.sum + dram__bytes_write.sum over one launch, divided by the
+# elements of that launch); the capture is summarised under profiles/.
+NCU_TRAFFIC_BYTES_PER_ELEMENT = {
+}
+
+
+def _peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        try:
+            with open(path) as f:
+                return float(json.load(f)["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return FALLBACK_HBM_GBS, "fallback"
+
+
+# --------------------------------------------------------------------------- clocks
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the GPU is under load."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.samples = []          # (t, sm, max, reasons[4])
+        self.proc = None
+        self.thread = None
+        self.gpu = gpu_index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.gpu}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                self.samples.append((time.time(), float(parts[0]), float(parts[1]), parts[3:7]))
+            except ValueError:
+                continue
+
+    def stop(self):
+        if self.proc is not None:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except Exception:
+                self.proc.kill()
+
+    def summary(self, t0: float, t1: float, window: str):
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        inside = [s for s in self.samples if t0 <= s[0] <= t1]
+        if not inside:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0, "window": window}
+        reasons = sorted({n for s in inside for n, v in zip(names, s[3]) if v.lower().startswith("active")})
+        return {"sm_mhz": statistics.median(s[1] for s in inside), "sm_max_mhz": max(s[2] for s in inside),
+                "reasons": reasons, "samples": len(inside), "window": window}
+
+
+# --------------------------------------------------------------------------- reference arm (the oracle on host cores)
+
+def _oracle_sample_rate(kinds, dtype, x_std, g_std, budget_s: float, threads: int):
+    """elements/s of the fp64 oracle (forward + rounding + backward) on a bounded sample."""
+    import numpy as np
+    import oracle
+    from paper_2209_10778_b200 import workloads as W
+    oracle.set_threads(threads)
+    n_probe = 1 << 18
+    x = W.raw_numpy(W.normal(n_probe, dtype, 0, x_std))
+    g = W.raw_numpy(W.normal(n_probe, dtype, 1, g_std))
+    t = time.perf_counter()
+    for k in kinds:
+        oracle.forward_backward(k, dtype, x, g)
+    probe = time.perf_counter() - t
+    rate = n_probe * len(kinds) / max(probe, 1e-9)
+    n = int(min(max(rate * budget_s / len(kinds), n_probe), 1 << 26))
+    x = W.raw_numpy(W.normal(n, dtype, 0, x_std))
+    g = W.raw_numpy(W.normal(n, dtype, 1, g_std))
+    t = time.perf_counter()
+    for k in kinds:
+        oracle.forward_backward(k, dtype, x, g)
+    dt = time.perf_counter() - t
+    return n * len(kinds) / dt, n, dt
+
+
+def run_reference(args, w):
+    """--impl reference: the oracle, as it stands, timed on the host cores.  Each step is
+    one fwd+round+bwd pass over a bounded sample, sized so that warm-up plus K steps take
+    about two minutes in all."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    from paper_2209_10778_b200 import workloads as W
+    threads = oracle.max_threads()
+    oracle.set_threads(threads)
+    probe_rate, _, _ = _oracle_sample_rate(w.kinds, w.dtype, w.x_std, w.g_std, 1.0, threads)
+    total = max(1, args.steps + args.warmup)
+    n_s = int(min(max(probe_rate * 120.0 / total / len(w.kinds), 4096), w.numel(0)))
+    x = W.raw_numpy(W.normal(n_s, w.dtype, w.x_seed, w.x_std))
+    g = W.raw_numpy(W.normal(n_s, w.dtype, w.g_seed, w.g_std))
+    times = []
+    for i in range(total):
+        t = time.perf_counter()
+        for k in w.kinds:
+            oracle.forward_backward(k, w.dtype, x, g)
+        if i >= args.warmup:
+            times.append(time.perf_counter() - t)
+    dt = sum(times)
+    value = n_s * len(w.kinds) * len(times) / dt if dt > 0 else 0.0
+    n_total = w.numel(0) * len(w.kinds)
+    sample = f"first {n_s} of {w.numel(0)} elements per kind, {len(w.kinds)} kinds, fwd+round+bwd in fp64, per step"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": (n_total / value * 1e3) if value else None, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": w.dtype, "data": "synthetic",
+        "config": {"workload": w.name, "kinds": list(w.kinds), "shape": list(w.shapes[0]),
+                   "note": "ms_per_step is the sample rate extrapolated to the full workload"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# --------------------------------------------------------------------------- our arm
+
+def run_ours(args, w):
+    import torch
+    import torch.distributed as dist
+    from paper_2209_10778_b200 import binding as nfad
+    from paper_2209_10778_b200 import workloads as W
+
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the path has no CPU implementation")
+    nfad.load()                                    # fails loudly if libnfad.so is missing
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    n = w.numel(0)
+    es = 4 if w.dtype == "f32" else 2
+    kinds = list(w.kinds)
+    per_set = 5 * n * es
+    n_sets = max(4, -(-4 * L2_BYTES // per_set) + 1)
+    n_sets += n_sets % 2
+    half = n_sets // 2
+
+    sets = []
+    for i in range(n_sets):
+        x = W.normal(n, w.dtype, w.x_seed + 100 * i, w.x_std, dev)
+        g = W.normal(n, w.dtype, w.g_seed + 100 * i, w.g_std, dev)
+        sets.append({"x": x, "g": g, "y": torch.empty_like(x), "d": torch.empty_like(x), "gin": torch.empty_like(x)})
+    for s in sets:                                  # every f' buffer holds a real derivative before timing
+        nfad.nfad_act_forward(kinds[0], s["x"], s["y"], s["d"])
+    torch.cuda.synchronize()
+
+    ev = {"fwd": [], "bwd": []}
+
+    def step(i: int, timed: bool):
+        for j, kind in enumerate(kinds):
+            a = sets[(len(kinds) * i + j) % n_sets]
+            b = sets[(len(kinds) * i + j + half) % n_sets]
+            if timed:
+                e0, e1, e2, e3 = (torch.cuda.Event(enable_timing=True) for _ in range(4))
+                e0.record()
+                nfad.nfad_act_forward(kind, a["x"], a["y"], a["d"])
+                e1.record()
+                e2.record()
+                nfad.nfad_act_backward(kind, b["g"], b["d"], b["gin"])
+                e3.record()
+                if j == 0:
+                    ev["fwd"].append((e0, e1))
+                    ev["bwd"].append((e2, e3))
+            else:
+                nfad.nfad_act_forward(kind, a["x"], a["y"], a["d"])
+                nfad.nfad_act_backward(kind, b["g"], b["d"], b["gin"])
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    if sampler:
+        sampler.start()
+    warm = max(3, args.warmup)
+    for i in range(warm):
+        step(i, False)
+    barrier()
+    t_wall0 = time.time()
+    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    start.record()
+    for i in range(args.steps):
+        step(warm + i, True)
+    end.record()
+    barrier()
+    t_wall1 = time.time()
+    ms = start.elapsed_time(end)
+    window = "timed region"
+    if sampler and (t_wall1 - t_wall0) < 1.5:
+        # the timed region is shorter than nvidia-smi's sampling period: keep the same loop
+        # running, untimed, so that the clock record is taken under the same load
+        window = "untimed continuation of the same loop (timed region < 1.5 s)"
+        t_wall0 = time.time()
+        i = 0
+        while time.time() - t_wall0 < 1.5:
+            for _ in range(50):
+                step(i, False)
+                i += 1
+            torch.cuda.synchronize()
+        t_wall1 = time.time()
+    if sampler:
+        sampler.stop()
+    if world > 1:
+        t = torch.tensor([ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+
+    fwd_ms = statistics.mean(a.elapsed_time(b) for a, b in ev["fwd"]) if ev["fwd"] else None
+    bwd_ms = statistics.mean(a.elapsed_time(b) for a, b in ev["bwd"]) if ev["bwd"] else None
+
+    # ---- end to end: host buffers in, host buffers out, copies inside the timed region
+    hx = [torch.empty(n, dtype=sets[0]["x"].dtype).pin_memory() for _ in kinds]
+    hg = [torch.empty(n, dtype=sets[0]["x"].dtype).pin_memory() for _ in kinds]
+    hy = [torch.empty(n, dtype=sets[0]["x"].dtype).pin_memory() for _ in kinds]
+    hgin = [torch.empty(n, dtype=sets[0]["x"].dtype).pin_memory() for _ in kinds]
+    for j in range(len(kinds)):
+        hx[j].copy_(sets[j]["x"])
+        hg[j].copy_(sets[j]["g"])
+
+    def e2e_step(i: int):
+        for j, kind in enumerate(kinds):
+            s = sets[(len(kinds) * i + j) % n_sets]
+            s["x"].copy_(hx[j], non_blocking=True)
+            s["g"].copy_(hg[j], non_blocking=True)
+            nfad.nfad_act_forward(kind, s["x"], s["y"], s["d"])
+            nfad.nfad_act_backward(kind, s["g"], s["d"], s["gin"])
+            hy[j].copy_(s["y"], non_blocking=True)
+            hgin[j].copy_(s["gin"], non_blocking=True)
+
+    e2e_steps = max(3, min(args.steps, 20))
+    for i in range(3):
+        e2e_step(i)
+    barrier()
+    s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    s0.record()
+    for i in range(e2e_steps):
+        e2e_step(i)
+    s1.record()
+    barrier()
+    e2e_ms = s0.elapsed_time(s1)
+    if world > 1:
+        t = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    elems_per_step = n * len(kinds)
+    value = world * elems_per_step * args.steps / (ms / 1e3)
+    e2e_value = world * elems_per_step * e2e_steps / (e2e_ms / 1e3)
+    peak, peak_kind = _peaks()
+    algo_bytes = 3 * es * n                       # forward: read x, write y and f'
+    achieved = algo_bytes / (fwd_ms / 1e3) / 1e9 if fwd_ms else None
+    key = f"{kinds[0]}_{w.dtype}_forward"
+    tpe = NCU_TRAFFIC_BYTES_PER_ELEMENT.get(key)
+    roofline = {
+        "bound": "hbm", "kernel": f"nfad_act_forward[{kinds[0]},{w.dtype}]", "achieved": achieved, "peak": peak,
+        "unit": "GB/s", "frac": (achieved / peak) if achieved else None, "peak_source": f"{peak_kind} copy bandwidth",
+        "frac_of_nominal_8000": (achieved / 8000.0) if achieved else None,
+        "algorithmic_bytes_per_launch": algo_bytes, "avg_launch_ms": fwd_ms,
+        "traffic": (tpe * n) if tpe else None,
+        "backward": {"achieved": (3 * es * n / (bwd_ms / 1e3) / 1e9) if bwd_ms else None, "avg_launch_ms": bwd_ms},
+    }
+
+    threads = 1
+    cpu_baseline = None
+    try:
+        import oracle
+        threads = oracle.max_threads()
+        rate, n_used, dt = _oracle_sample_rate(kinds, w.dtype, w.x_std, w.g_std, 10.0, threads)
+        cpu_baseline = {"value": rate, "unit": UNIT, "cores": threads, "kind": "oracle",
+                        "sample": f"first {n_used} of {n} elements per kind, {len(kinds)} kinds, {dt:.1f} s"}
+    except Exception as exc:  # the oracle is test infrastructure; its absence must not hide the GPU number
+        cpu_baseline = {"value": None, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": f"unavailable: {exc}"}
+
+    saved = {lay: nfad.nfad_saved_bytes_per_element(kinds[0], w.dtype, lay) for lay in nfad.LAYOUTS}
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": warm,
+        "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": w.dtype, "data": "synthetic",
+        "config": {"workload": w.name, "kinds": kinds, "shape": list(w.shapes[0]), "elements": n,
+                   "l2": f"{n_sets} rotating buffer sets ({n_sets * per_set >> 20} MiB), backward reads the f' written "
+                         f"{half} sets earlier: no tensor is re-used from L2",
+                   "saved_bytes_per_element": saved},
+        "roofline": roofline, "cpu_baseline": cpu_baseline,
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": 2 * n * es * len(kinds),
+                "d2h_bytes_per_step": 2 * n * es * len(kinds), "steps": e2e_steps},
+        "gpu_launches": 2 * len(kinds) * args.steps,
+        "clocks": sampler.summary(t_wall0, t_wall1, window) if sampler else None,
+    }
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="bert_base_ffn")
+    args = ap.parse_args()
+    from paper_2209_10778_b200 import workloads as W
+    w = W.WORKLOADS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, w)
+    else:
+        run_ours(args, w)
+
+
+if __name__ == "__main__":
+    main()

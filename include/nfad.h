@@ -1,0 +1,164 @@
+/*
+ * nfad.h -- C interface of the nested Forward-AD activation library (CUDA, sm_100a).
+ *
+ * The method (Section II-C approach 3, Section II-E): an element-wise activation
+ * f is evaluated once, in the forward pass, on dual numbers (value, tangent)
+ * seeded with tangent 1 (Section II-D), so that the forward pass emits y = f(x)
+ * and f'(x) together; f'(x) is the ONLY tensor kept for back-propagation, and
+ * the backward pass is the single multiplication grad_in = grad_out * f'(x)
+ * (Eq. 4; "replaces the BFN with a direct Multiplication", Section IV).
+ *
+ * Conventions common to every entry point
+ *   - Every tensor argument is a DEVICE pointer to a flat, contiguous array of n
+ *     elements of `dtype` (NFAD_F32: float; NFAD_BF16: bfloat16; NFAD_F16: IEEE
+ *     half).  Tensor shape is irrelevant to an element-wise pass.  The caller
+ *     owns all memory; the library allocates none and keeps no state between
+ *     calls.  Arithmetic is fp32 for every storage type; results are rounded to
+ *     nearest-even once, at the store.  Subnormals are kept (no flush to zero).
+ *   - Pointers need only the natural alignment of `dtype`.  When all tensors of
+ *     a call share one offset modulo 16 bytes the 128-bit path is used (elements
+ *     before the first and after the last whole 16-byte packet are handled one
+ *     by one); otherwise every element is handled one by one.  Results do not
+ *     depend on the path.
+ *   - Exact in-place use (an output pointer equal to an input pointer) is
+ *     allowed.  Two outputs that overlap, or an output that overlaps an input
+ *     without being equal to it, give NFAD_E_OVERLAP.
+ *   - Work is enqueued on `stream` (a cudaStream_t; 0 is the legacy default
+ *     stream) of the current device and the call returns at once.  The return
+ *     value covers argument validation and the launch, not completion.
+ *   - n == 0 is valid and does nothing.  n is 64-bit: 2^30 fp32 elements and
+ *     beyond are indexed correctly.
+ *   - Return value: an nfad_status.  Nothing aborts or traps.  After
+ *     NFAD_E_CUDA, nfad_last_cuda_error() gives the cudaError_t of the calling
+ *     thread's failed call.
+ *   - Non-finite input: NaN gives NaN in y and f'.  +inf gives y = +inf,
+ *     f' = 1; -inf gives y = -0, f' = +-0.
+ */
+#ifndef NFAD_H_
+#define NFAD_H_
+
+#include <stddef.h>
+
+#if defined(__GNUC__)
+#define NFAD_API __attribute__((visibility("default")))
+#else
+#define NFAD_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* Activations: Table I (GELU in its tanh form, Mish, Swish) and the erf-exact
+ * GELU x*Phi(x) that Table I's tanh form approximates.  The two GELUs are
+ * different functions (they differ by up to ~5e-4) and are never interchanged. */
+typedef enum {
+    NFAD_GELU_ERF = 0,   /* x * (1 + erf(x / sqrt 2)) / 2                                  */
+    NFAD_GELU_TANH = 1,  /* 0.5 x (1 + tanh( sqrt(2/pi) (x + 0.044715 x^3) ))   (Table I)  */
+    NFAD_SWISH = 2,      /* x * sigmoid(x)                                       (Table I)  */
+    NFAD_MISH = 3        /* x * tanh(softplus(x))                                (Table I)  */
+} nfad_kind;
+
+typedef enum { NFAD_F32 = 0, NFAD_BF16 = 1, NFAD_F16 = 2 } nfad_dtype;
+
+typedef enum {
+    NFAD_OK = 0,
+    NFAD_E_KIND = 1,     /* kind is not an nfad_kind                                  */
+    NFAD_E_DTYPE = 2,    /* dtype is not an nfad_dtype                                */
+    NFAD_E_NULL = 3,     /* a tensor pointer is NULL while n > 0                      */
+    NFAD_E_OVERLAP = 4,  /* forbidden aliasing, see above                             */
+    NFAD_E_CUDA = 5,     /* a CUDA call failed: see nfad_last_cuda_error()            */
+    NFAD_E_ALIGN = 6,    /* a pointer is not a multiple of the element size           */
+    NFAD_E_SCRATCH = 7,  /* scratch_bytes is smaller than the comparator needs        */
+    NFAD_E_LAYOUT = 8    /* layout is not an nfad_layout                              */
+} nfad_status;
+
+/* How the tensor needed by backward is kept between the passes (Section II-C). */
+typedef enum {
+    NFAD_LAYOUT_NESTED = 0,     /* approach 3: keep f'(x)                                         */
+    NFAD_LAYOUT_CONVENTIONAL = 1, /* keep x; one fused backward kernel re-derives f'(x)           */
+    NFAD_LAYOUT_RECOMPUTE = 2,  /* approach 2: keep x; backward re-runs the forward operators     */
+    NFAD_LAYOUT_OP_BY_OP = 3    /* approach 1: every operator keeps what its own rule needs       */
+} nfad_layout;
+
+typedef void* nfad_stream_t;   /* a cudaStream_t */
+
+/*
+ * Forward pass of the nested method (Section II-C approach 3; Eq. 3 for the
+ * product rule that merges the tangents; Section II-D for the seed x' = 1).
+ *   x     [in]  n elements
+ *   y     [out] n elements, y[i] = f(x[i])
+ *   dfdx  [out] n elements, dfdx[i] = f'(x[i]): the tensor to keep for backward
+ * y may equal x (in place).  dfdx may equal x.  y and dfdx must not overlap.
+ */
+NFAD_API int nfad_act_forward(int kind, int dtype, const void* x, void* y, void* dfdx, size_t n, nfad_stream_t stream);
+
+/*
+ * Forward pass without the tangent (inference, or any pass that will not be
+ * differentiated): the same chain of primitives, value parts only.
+ *   x [in] n elements;  y [out] n elements (may equal x).
+ */
+NFAD_API int nfad_act_forward_infer(int kind, int dtype, const void* x, void* y, size_t n, nfad_stream_t stream);
+
+/*
+ * Backward pass of the nested method (Eq. 4, Section II-E): one multiplication,
+ *   grad_in[i] = round( grad_out[i] * dfdx[i] ),
+ * the product formed exactly and rounded once.  `kind` is validated but does
+ * not change the result.  grad_in may equal grad_out or dfdx.
+ */
+NFAD_API int nfad_act_backward(int kind, int dtype, const void* grad_out, const void* dfdx, void* grad_in, size_t n,
+                      nfad_stream_t stream);
+
+/*
+ * Comparator, conventional layout: the forward pass is nfad_act_forward_infer and
+ * x itself is kept; this backward re-derives f'(x) from x with the whole
+ * transcendental chain and multiplies, in one kernel (f' is not rounded to the
+ * storage type on the way):  grad_in[i] = round( grad_out[i] * f'(x[i]) ).
+ * grad_in may equal grad_out or x.
+ */
+NFAD_API int nfad_cmp_conv_backward(int kind, int dtype, const void* grad_out, const void* x, void* grad_in, size_t n,
+                           nfad_stream_t stream);
+
+/*
+ * Comparator, recomputation layout (Section II-C approach 2): x is kept; backward
+ * runs two kernels.  The first re-runs the forward operators and writes the
+ * intermediate that the per-operator backward rules need (the gate h(x) of
+ * f = x h(x): sigmoid(x) for Swish, i.e. v1 of the paper's example) to `scratch`
+ * in the storage type; the second reads grad_out, x and that intermediate and
+ * walks the rules of Eqs. 1-2: grad_in = g h + g x h'.
+ *   scratch [scratch] at least nfad_cmp_recompute_scratch_bytes(kind, dtype, n)
+ *           bytes of device memory, 16-byte aligned; contents undefined after.
+ * Accuracy is that of operator-by-operator back-propagation through a stored
+ * intermediate (1 - h is formed by subtraction), not that of the nested path.
+ * grad_in may equal grad_out; it must not overlap x or scratch.
+ */
+NFAD_API int nfad_cmp_recompute_backward(int kind, int dtype, const void* grad_out, const void* x, void* scratch,
+                                size_t scratch_bytes, void* grad_in, size_t n, nfad_stream_t stream);
+
+/* Bytes of scratch the recomputation comparator needs for n elements; 0 on a bad kind or dtype. */
+NFAD_API size_t nfad_cmp_recompute_scratch_bytes(int kind, int dtype, size_t n);
+
+/*
+ * Bytes per element that a layout keeps alive between the forward and the
+ * backward pass.  Nested, conventional and recomputation keep one tensor;
+ * operator-by-operator back-propagation keeps every tensor its rules need
+ * (for Swish the paper's own count, x and sigmoid(x), Section II-C approach 1;
+ * for the other kinds the count under the usual per-operator rules).
+ * Returns a negative nfad_status on a bad argument.
+ */
+NFAD_API int nfad_saved_bytes_per_element(int kind, int dtype, int layout);
+
+/* The cudaError_t (as an int) behind the calling thread's last NFAD_E_CUDA; 0 if none. */
+NFAD_API int nfad_last_cuda_error(void);
+
+/* A static, human-readable name for a status. */
+NFAD_API const char* nfad_status_string(int status);
+
+/* Library version, "major.minor.patch". */
+NFAD_API const char* nfad_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+
+#endif /* NFAD_H_ */

@@ -1,0 +1,12 @@
+"""Nested Forward-AD activation pass for B200 (sm_100a).
+
+``binding`` mirrors the C interface of ``libnfad.so`` (see ``include/nfad.h``);
+``workloads`` draws the seeded synthetic inputs; ``build`` compiles the library.
+"""
+from . import workloads  # noqa: F401
+from .binding import (  # noqa: F401
+    DTYPES, KINDS, LAYOUTS, NfadError, load,
+    nfad_act_backward, nfad_act_forward, nfad_act_forward_infer,
+    nfad_cmp_conv_backward, nfad_cmp_recompute_backward, nfad_cmp_recompute_scratch_bytes,
+    nfad_saved_bytes_per_element, nfad_status_string, nfad_version,
+)

@@ -1,0 +1,165 @@
+"""Thin ctypes binding over libnfad.so: same names as the C interface
+(``include/nfad.h``), argument marshalling only.  Every step of the path runs
+in the library's CUDA kernels; there is no fallback of any kind: if the
+library cannot be loaded, or a tensor is not a contiguous CUDA tensor of a
+supported type, the call raises.
+
+PyTorch appears here only as the owner of device memory and streams.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import torch
+
+KINDS = {"gelu_erf": 0, "gelu_tanh": 1, "swish": 2, "mish": 3}
+DTYPES = {"f32": 0, "bf16": 1, "f16": 2}
+LAYOUTS = {"nested": 0, "conventional": 1, "recompute": 2, "op_by_op": 3}
+_TORCH_TO_CODE = {torch.float32: 0, torch.bfloat16: 1, torch.float16: 2}
+
+NFAD_OK = 0
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libnfad.so")
+
+EXPORTS = (
+    "nfad_act_forward", "nfad_act_forward_infer", "nfad_act_backward",
+    "nfad_cmp_conv_backward", "nfad_cmp_recompute_backward", "nfad_cmp_recompute_scratch_bytes",
+    "nfad_saved_bytes_per_element", "nfad_last_cuda_error", "nfad_status_string", "nfad_version",
+)
+
+_lib: Optional[ctypes.CDLL] = None
+
+
+class NfadError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        lib = load()
+        msg = lib.nfad_status_string(status).decode()
+        if status == 5:
+            msg += f" [cudaError {lib.nfad_last_cuda_error()}]"
+        super().__init__(f"{where}: {msg} (status {status})")
+
+
+def load() -> ctypes.CDLL:
+    """Loads libnfad.so from the package directory.  Raises if it has not been built
+    (``python -m paper_2209_10778_b200.build``): nothing else can run the path."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2209_10778_b200.build` "
+                              "(needs nvcc); there is no other implementation of the path")
+        lib = ctypes.CDLL(LIB_PATH)
+        vp, sz, ci = ctypes.c_void_p, ctypes.c_size_t, ctypes.c_int
+        lib.nfad_act_forward.argtypes = [ci, ci, vp, vp, vp, sz, vp]
+        lib.nfad_act_forward_infer.argtypes = [ci, ci, vp, vp, sz, vp]
+        lib.nfad_act_backward.argtypes = [ci, ci, vp, vp, vp, sz, vp]
+        lib.nfad_cmp_conv_backward.argtypes = [ci, ci, vp, vp, vp, sz, vp]
+        lib.nfad_cmp_recompute_backward.argtypes = [ci, ci, vp, vp, vp, sz, vp, sz, vp]
+        lib.nfad_cmp_recompute_scratch_bytes.argtypes = [ci, ci, sz]
+        lib.nfad_cmp_recompute_scratch_bytes.restype = sz
+        lib.nfad_saved_bytes_per_element.argtypes = [ci, ci, ci]
+        lib.nfad_last_cuda_error.argtypes = []
+        lib.nfad_status_string.argtypes = [ci]
+        lib.nfad_status_string.restype = ctypes.c_char_p
+        lib.nfad_version.argtypes = []
+        lib.nfad_version.restype = ctypes.c_char_p
+        for name in ("nfad_act_forward", "nfad_act_forward_infer", "nfad_act_backward", "nfad_cmp_conv_backward",
+                     "nfad_cmp_recompute_backward", "nfad_saved_bytes_per_element", "nfad_last_cuda_error"):
+            getattr(lib, name).restype = ci
+        _lib = lib
+    return _lib
+
+
+def _kind(kind) -> int:
+    return KINDS[kind] if isinstance(kind, str) else int(kind)
+
+
+def _tensor(t: torch.Tensor, name: str, like: Optional[torch.Tensor] = None) -> int:
+    if not isinstance(t, torch.Tensor) or not t.is_cuda:
+        raise TypeError(f"{name} must be a CUDA tensor")
+    if t.dtype not in _TORCH_TO_CODE:
+        raise TypeError(f"{name}: unsupported dtype {t.dtype}")
+    if not t.is_contiguous():
+        raise ValueError(f"{name} must be contiguous")
+    if like is not None and (t.dtype != like.dtype or t.numel() != like.numel() or t.device != like.device):
+        raise ValueError(f"{name} must match the first tensor's dtype, size and device")
+    return t.data_ptr()
+
+
+def _stream(t: torch.Tensor) -> int:
+    return torch.cuda.current_stream(t.device).cuda_stream
+
+
+def _check(rc: int, where: str) -> None:
+    if rc != NFAD_OK:
+        raise NfadError(rc, where)
+
+
+def nfad_act_forward(kind, x: torch.Tensor, y: torch.Tensor, dfdx: torch.Tensor) -> None:
+    """x -> (y = f(x), dfdx = f'(x)), one kernel on the current stream."""
+    px = _tensor(x, "x")
+    with torch.cuda.device(x.device):
+        _check(load().nfad_act_forward(_kind(kind), _TORCH_TO_CODE[x.dtype], px, _tensor(y, "y", x),
+                                       _tensor(dfdx, "dfdx", x), x.numel(), _stream(x)), "nfad_act_forward")
+
+
+def nfad_act_forward_infer(kind, x: torch.Tensor, y: torch.Tensor) -> None:
+    px = _tensor(x, "x")
+    with torch.cuda.device(x.device):
+        _check(load().nfad_act_forward_infer(_kind(kind), _TORCH_TO_CODE[x.dtype], px, _tensor(y, "y", x),
+                                             x.numel(), _stream(x)), "nfad_act_forward_infer")
+
+
+def nfad_act_backward(kind, grad_out: torch.Tensor, dfdx: torch.Tensor, grad_in: torch.Tensor) -> None:
+    """grad_in = grad_out * dfdx (one rounding)."""
+    pg = _tensor(grad_out, "grad_out")
+    with torch.cuda.device(grad_out.device):
+        _check(load().nfad_act_backward(_kind(kind), _TORCH_TO_CODE[grad_out.dtype], pg, _tensor(dfdx, "dfdx", grad_out),
+                                        _tensor(grad_in, "grad_in", grad_out), grad_out.numel(), _stream(grad_out)),
+               "nfad_act_backward")
+
+
+def nfad_cmp_conv_backward(kind, grad_out: torch.Tensor, x: torch.Tensor, grad_in: torch.Tensor) -> None:
+    pg = _tensor(grad_out, "grad_out")
+    with torch.cuda.device(grad_out.device):
+        _check(load().nfad_cmp_conv_backward(_kind(kind), _TORCH_TO_CODE[grad_out.dtype], pg, _tensor(x, "x", grad_out),
+                                             _tensor(grad_in, "grad_in", grad_out), grad_out.numel(), _stream(grad_out)),
+               "nfad_cmp_conv_backward")
+
+
+def nfad_cmp_recompute_scratch_bytes(kind, dtype, n: int) -> int:
+    code = DTYPES[dtype] if isinstance(dtype, str) else _TORCH_TO_CODE[dtype]
+    return int(load().nfad_cmp_recompute_scratch_bytes(_kind(kind), code, n))
+
+
+def nfad_cmp_recompute_backward(kind, grad_out: torch.Tensor, x: torch.Tensor, scratch: torch.Tensor,
+                                grad_in: torch.Tensor) -> None:
+    """scratch: any contiguous CUDA tensor with at least nfad_cmp_recompute_scratch_bytes bytes."""
+    pg = _tensor(grad_out, "grad_out")
+    if not scratch.is_cuda or not scratch.is_contiguous():
+        raise TypeError("scratch must be a contiguous CUDA tensor")
+    with torch.cuda.device(grad_out.device):
+        _check(load().nfad_cmp_recompute_backward(_kind(kind), _TORCH_TO_CODE[grad_out.dtype], pg, _tensor(x, "x", grad_out),
+                                                  scratch.data_ptr(), scratch.numel() * scratch.element_size(),
+                                                  _tensor(grad_in, "grad_in", grad_out), grad_out.numel(),
+                                                  _stream(grad_out)), "nfad_cmp_recompute_backward")
+
+
+def nfad_saved_bytes_per_element(kind, dtype, layout) -> int:
+    code = DTYPES[dtype] if isinstance(dtype, str) else _TORCH_TO_CODE[dtype]
+    lay = LAYOUTS[layout] if isinstance(layout, str) else int(layout)
+    rc = load().nfad_saved_bytes_per_element(_kind(kind), code, lay)
+    if rc < 0:
+        raise NfadError(-rc, "nfad_saved_bytes_per_element")
+    return rc
+
+
+def nfad_version() -> str:
+    return load().nfad_version().decode()
+
+
+def nfad_status_string(status: int) -> str:
+    return load().nfad_status_string(int(status)).decode()

@@ -1,0 +1,181 @@
+// nfad_api.cu -- the extern "C" boundary: argument validation, aliasing rules,
+// and dispatch to the per-storage-type launchers.  No arithmetic lives here.
+#include <stdint.h>
+
+#include "../../include/nfad.h"
+#include "nfad_internal.h"
+
+namespace {
+
+thread_local int g_last_cuda_error = 0;
+
+size_t elem_size(int dtype) { return dtype == NFAD_F32 ? 4 : 2; }
+
+bool overlaps(const void* a, const void* b, size_t bytes_a, size_t bytes_b)
+{
+    uintptr_t a0 = reinterpret_cast<uintptr_t>(a), b0 = reinterpret_cast<uintptr_t>(b);
+    return a0 < b0 + bytes_b && b0 < a0 + bytes_a;
+}
+
+// Validates the tensors of one launch.  Inputs may be exactly equal to outputs;
+// any other overlap that involves an output is rejected.
+int check(int kind, int dtype, const void* const* in, int nin, void* const* out, int nout, size_t n)
+{
+    if (kind < 0 || kind > 3) return NFAD_E_KIND;
+    if (dtype < 0 || dtype > 2) return NFAD_E_DTYPE;
+    if (n == 0) return NFAD_OK;
+    const size_t es = elem_size(dtype), bytes = n * es;
+    for (int i = 0; i < nin; ++i) {
+        if (!in[i]) return NFAD_E_NULL;
+        if (reinterpret_cast<uintptr_t>(in[i]) % es) return NFAD_E_ALIGN;
+    }
+    for (int i = 0; i < nout; ++i) {
+        if (!out[i]) return NFAD_E_NULL;
+        if (reinterpret_cast<uintptr_t>(out[i]) % es) return NFAD_E_ALIGN;
+    }
+    for (int i = 0; i < nout; ++i) {
+        for (int j = i + 1; j < nout; ++j)
+            if (overlaps(out[i], out[j], bytes, bytes)) return NFAD_E_OVERLAP;
+        for (int j = 0; j < nin; ++j)
+            if (in[j] != out[i] && overlaps(out[i], in[j], bytes, bytes)) return NFAD_E_OVERLAP;
+    }
+    return NFAD_OK;
+}
+
+int run(nfad::OpCode op, int kind, int dtype, const void* const* in, void* const* out, size_t n, nfad_stream_t stream)
+{
+    if (n == 0) return NFAD_OK;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaError_t e = dtype == NFAD_F32 ? nfad::launch_f32(op, kind, in, out, n, st)
+                                      : nfad::launch_16(op, kind, dtype, in, out, n, st);
+    if (e != cudaSuccess) {
+        g_last_cuda_error = static_cast<int>(e);
+        return NFAD_E_CUDA;
+    }
+    return NFAD_OK;
+}
+
+// Tensors kept by operator-by-operator back-propagation under the usual rules
+// (mul keeps both operands; tanh / sigmoid keep their output; erf / softplus
+// keep their input; add and scale-by-constant keep nothing).
+//   Swish     mul(x, sigmoid x)                      {x, sigmoid}           = 2  (the paper's v1, v2)
+//   Mish      mul(x, tanh(softplus x))               {x, tanh}              = 2
+//   GELU-tanh mul(0.5 x, 1 + tanh(c (x + a x^3)))    {x, 0.5x, tanh, 1+tanh} = 4
+//   GELU-erf  mul(0.5 x, 1 + erf(x / sqrt2))         {x/sqrt2, 0.5x, 1+erf} = 3
+int op_by_op_tensors(int kind)
+{
+    switch (kind) {
+    case NFAD_SWISH: return 2;
+    case NFAD_MISH: return 2;
+    case NFAD_GELU_TANH: return 4;
+    default: return 3;
+    }
+}
+
+}  // namespace
+
+extern "C" {
+
+int nfad_act_forward(int kind, int dtype, const void* x, void* y, void* dfdx, size_t n, nfad_stream_t stream)
+{
+    const void* in[1] = {x};
+    void* out[2] = {y, dfdx};
+    int rc = check(kind, dtype, in, 1, out, 2, n);
+    return rc ? rc : run(nfad::kOpForward, kind, dtype, in, out, n, stream);
+}
+
+int nfad_act_forward_infer(int kind, int dtype, const void* x, void* y, size_t n, nfad_stream_t stream)
+{
+    const void* in[1] = {x};
+    void* out[1] = {y};
+    int rc = check(kind, dtype, in, 1, out, 1, n);
+    return rc ? rc : run(nfad::kOpForwardInfer, kind, dtype, in, out, n, stream);
+}
+
+int nfad_act_backward(int kind, int dtype, const void* grad_out, const void* dfdx, void* grad_in, size_t n,
+                      nfad_stream_t stream)
+{
+    const void* in[2] = {grad_out, dfdx};
+    void* out[1] = {grad_in};
+    int rc = check(kind, dtype, in, 2, out, 1, n);
+    return rc ? rc : run(nfad::kOpBackward, kind, dtype, in, out, n, stream);
+}
+
+int nfad_cmp_conv_backward(int kind, int dtype, const void* grad_out, const void* x, void* grad_in, size_t n,
+                           nfad_stream_t stream)
+{
+    const void* in[2] = {grad_out, x};
+    void* out[1] = {grad_in};
+    int rc = check(kind, dtype, in, 2, out, 1, n);
+    return rc ? rc : run(nfad::kOpConvBackward, kind, dtype, in, out, n, stream);
+}
+
+size_t nfad_cmp_recompute_scratch_bytes(int kind, int dtype, size_t n)
+{
+    if (kind < 0 || kind > 3 || dtype < 0 || dtype > 2) return 0;
+    size_t b = n * elem_size(dtype);
+    return (b + 15) & ~size_t(15);
+}
+
+int nfad_cmp_recompute_backward(int kind, int dtype, const void* grad_out, const void* x, void* scratch,
+                                size_t scratch_bytes, void* grad_in, size_t n, nfad_stream_t stream)
+{
+    if (kind < 0 || kind > 3) return NFAD_E_KIND;
+    if (dtype < 0 || dtype > 2) return NFAD_E_DTYPE;
+    if (n == 0) return NFAD_OK;
+    if (!scratch) return NFAD_E_NULL;
+    if (scratch_bytes < nfad_cmp_recompute_scratch_bytes(kind, dtype, n)) return NFAD_E_SCRATCH;
+    {
+        const void* in[1] = {x};
+        void* out[1] = {scratch};
+        int rc = check(kind, dtype, in, 1, out, 1, n);
+        if (rc) return rc;
+        if (x == scratch) return NFAD_E_OVERLAP;
+    }
+    const void* in2[3] = {grad_out, x, scratch};
+    void* out2[1] = {grad_in};
+    int rc = check(kind, dtype, in2, 3, out2, 1, n);
+    if (rc) return rc;
+    if (grad_in == x || grad_in == scratch) return NFAD_E_OVERLAP;
+    const void* in1[1] = {x};
+    void* out1[1] = {scratch};
+    rc = run(nfad::kOpRecompute1, kind, dtype, in1, out1, n, stream);
+    if (rc) return rc;
+    return run(nfad::kOpRecompute2, kind, dtype, in2, out2, n, stream);
+}
+
+int nfad_saved_bytes_per_element(int kind, int dtype, int layout)
+{
+    if (kind < 0 || kind > 3) return -NFAD_E_KIND;
+    if (dtype < 0 || dtype > 2) return -NFAD_E_DTYPE;
+    int s = static_cast<int>(elem_size(dtype));
+    switch (layout) {
+    case NFAD_LAYOUT_NESTED: return s;         // f'(x)
+    case NFAD_LAYOUT_CONVENTIONAL: return s;   // x
+    case NFAD_LAYOUT_RECOMPUTE: return s;      // x
+    case NFAD_LAYOUT_OP_BY_OP: return s * op_by_op_tensors(kind);
+    default: return -NFAD_E_LAYOUT;
+    }
+}
+
+int nfad_last_cuda_error(void) { return g_last_cuda_error; }
+
+const char* nfad_status_string(int status)
+{
+    switch (status) {
+    case NFAD_OK: return "ok";
+    case NFAD_E_KIND: return "unknown activation kind";
+    case NFAD_E_DTYPE: return "unknown storage dtype";
+    case NFAD_E_NULL: return "null tensor pointer";
+    case NFAD_E_OVERLAP: return "tensors overlap in a way that is not exact in-place use";
+    case NFAD_E_CUDA: return "CUDA error (see nfad_last_cuda_error)";
+    case NFAD_E_ALIGN: return "pointer not aligned to the element size";
+    case NFAD_E_SCRATCH: return "scratch buffer too small";
+    case NFAD_E_LAYOUT: return "unknown layout";
+    default: return "unknown status";
+    }
+}
+
+const char* nfad_version(void) { return "0.1.0"; }
+
+}  // extern "C"

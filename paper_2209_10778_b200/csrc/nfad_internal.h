@@ -1,0 +1,26 @@
+// nfad_internal.h -- launchers behind the C-ABI, one set per translation unit:
+// the fp32-storage kernels are built with floating-point contraction off (their
+// compensated arithmetic depends on it), the 16-bit-storage kernels with it on.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stddef.h>
+
+namespace nfad {
+
+enum Kind { kGeluErf = 0, kGeluTanh = 1, kSwish = 2, kMish = 3 };
+enum DType { kF32 = 0, kBF16 = 1, kF16 = 2 };
+
+// Which map to run.  Tensor order in `in` / `out` is fixed per op:
+//   kOpForward        in {x}            out {y, dfdx}
+//   kOpForwardInfer   in {x}            out {y}
+//   kOpBackward       in {g, dfdx}      out {gin}
+//   kOpConvBackward   in {g, x}         out {gin}
+//   kOpRecompute1     in {x}            out {h}
+//   kOpRecompute2     in {g, x, h}      out {gin}
+enum OpCode { kOpForward, kOpForwardInfer, kOpBackward, kOpConvBackward, kOpRecompute1, kOpRecompute2 };
+
+cudaError_t launch_f32(OpCode op, int kind, const void* const* in, void* const* out, size_t n, cudaStream_t st);
+cudaError_t launch_16(OpCode op, int kind, int dtype, const void* const* in, void* const* out, size_t n, cudaStream_t st);
+
+}  // namespace nfad

@@ -1,0 +1,122 @@
+// nfad_ops.cuh -- the per-element bodies that the streaming engine maps over
+// tensors: the nested Forward-AD forward and backward, and the two comparator
+// layouts that save x instead of f'(x).
+#pragma once
+
+#include "nfad_dual.cuh"
+
+namespace nfad {
+
+// Forward, training: x -> (y = f(x), f'(x)).  One pass over dual numbers; f'(x)
+// is the only tensor kept for back-propagation (Section II-C, approach 3).
+template <class K, class P> struct ForwardTrainOp {
+    static constexpr int kIn = 1, kOut = 2;
+    static __device__ __forceinline__ constexpr bool keep(int k) { return k == 0; }   // y is consumed next; f' much later
+    static __device__ __forceinline__ void apply(const float (&in)[1], float (&out)[2])
+    {
+        ActOut o = evaluate<K, P>(in[0]);
+        out[0] = o.y;
+        out[1] = o.dydx;
+    }
+};
+
+// Forward, inference: x -> y.  Same chain; the tangent parts are dead code.
+template <class K, class P> struct ForwardInferOp {
+    static constexpr int kIn = 1, kOut = 1;
+    static __device__ __forceinline__ constexpr bool keep(int) { return true; }
+    static __device__ __forceinline__ void apply(const float (&in)[1], float (&out)[1])
+    {
+        out[0] = evaluate<K, P>(in[0]).y;
+    }
+};
+
+// Backward of the nested layout (Eq. 4): grad_in = grad_out * f'(x), one multiply.
+// The fp32 product of two 16-bit values is exact unless it underflows; only bf16
+// shares fp32's exponent range, so only there can a product land below 2^-126,
+// where it is re-formed in fp64 and rounded straight to the bf16 subnormal grid
+// (multiples of 2^-133) to keep the result a single rounding of the true product.
+template <bool kBf16> struct BackwardOp {
+    static constexpr int kIn = 2, kOut = 1;
+    static __device__ __forceinline__ constexpr bool keep(int) { return true; }
+    static __device__ __forceinline__ void apply(const float (&in)[2], float (&out)[1])
+    {
+        float p = in[0] * in[1];
+        if (kBf16) {
+            if (fabsf(p) <= 1.17549435e-38f) {
+                const double kGrid = 6.2038417431289079e-25;   // 1.5 * 2^-81: ulp is 2^-133
+                double pd = (double)in[0] * (double)in[1];
+                pd = (pd + kGrid) - kGrid;
+                p = (float)pd;
+            }
+        }
+        out[0] = p;
+    }
+};
+
+// Conventional layout: x is saved, and backward re-derives f'(x) with the full
+// transcendental chain before the multiply.
+template <class K, class P> struct ConvBackwardOp {
+    static constexpr int kIn = 2, kOut = 1;
+    static __device__ __forceinline__ constexpr bool keep(int) { return true; }
+    static __device__ __forceinline__ void apply(const float (&in)[2], float (&out)[1])
+    {
+        out[0] = in[0] * evaluate<K, P>(in[1]).dydx;
+    }
+};
+
+// Recomputation layout (Section II-C, approach 2): x is saved; backward first
+// re-runs the forward operators to re-materialise the intermediate the
+// per-operator backward rules need (the gate h = v1 of the Swish example), then
+// walks those rules: x' = g v1 + g v2 v1' with v2 = x (Eq. 2).
+template <class K, class P> struct RecomputePhase1Op {
+    static constexpr int kIn = 1, kOut = 1;
+    static __device__ __forceinline__ constexpr bool keep(int) { return true; }
+    static __device__ __forceinline__ void apply(const float (&in)[1], float (&out)[1])
+    {
+        out[0] = evaluate_gate<K, P>(in[0]);
+    }
+};
+
+// h'(x) from x and the re-materialised h, by each operator's usual backward rule
+// (sigmoid: h(1-h); tanh: 1-t^2; erf: exp(-z^2) 2/sqrt(pi); softplus: sigmoid(x)).
+template <class K> struct GateSlope;
+template <> struct GateSlope<Swish> {
+    static __device__ __forceinline__ float of(float, float h) { return h * (1.0f - h); }
+};
+template <> struct GateSlope<GeluTanh> {
+    static __device__ __forceinline__ float of(float x, float h)
+    {
+        float du2 = fmaf(0.2140747458f, x * x, 1.5957691216f);     // 2 sqrt(2/pi) (1 + 3 * 0.044715 x^2)
+        return du2 * (h * (1.0f - h));
+    }
+};
+template <> struct GateSlope<GeluErf> {
+    static __device__ __forceinline__ float of(float x, float)
+    {
+        float xc = fminf(fabsf(x), 20.0f);
+        return 0.3989422804f * hw::ex2_approx(-0.72134752f * (xc * xc));   // phi(x)
+    }
+};
+template <> struct GateSlope<Mish> {
+    static __device__ __forceinline__ float of(float x, float t)
+    {
+        float xc = fminf(fabsf(x), 120.0f);
+        float e = hw::ex2_approx(-1.44269502f * xc);
+        float r = hw::rcp_approx(1.0f + e);
+        float sig = x < 0.0f ? e * r : r;
+        return fmaf(-t, t, 1.0f) * sig;
+    }
+};
+
+template <class K, class P> struct RecomputePhase2Op {
+    static constexpr int kIn = 3, kOut = 1;            // grad_out, x, h
+    static __device__ __forceinline__ constexpr bool keep(int) { return true; }
+    static __device__ __forceinline__ void apply(const float (&in)[3], float (&out)[1])
+    {
+        float g = in[0], x = in[1], h = in[2];
+        float hs = GateSlope<K>::of(x, h);
+        out[0] = fmaf(g * x, hs, g * h);
+    }
+};
+
+}  // namespace nfad

@@ -1,0 +1,294 @@
+// nfad_stream.cuh -- the HBM-streaming engine shared by every kernel of the
+// activation pass.  Each kernel is an element-wise map from NIN flat input
+// tensors to NOUT flat output tensors of one storage type; nothing is reused, so
+// the only jobs are (1) move 16-byte packets with fully coalesced accesses and
+// enough of them in flight to cover HBM latency, and (2) spend as few issue
+// slots per element as possible between the load and the store.
+//
+// Work decomposition: a tile is kBlock * kUnroll consecutive packets; thread t
+// of a CTA owns packets t, t + kBlock, ... of the tile, so every warp-level
+// access is one contiguous 512-byte run.  A grid of (SM count x resident CTAs)
+// walks the tiles with a grid stride; each thread issues all kUnroll * NIN loads
+// of its tile before the first use.  Elements before the first and after the
+// last whole packet (unaligned base, ragged tail) are handled one by one by the
+// first warps of CTA 0 with the very same per-element code, so the vector and
+// scalar paths agree bit for bit.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace nfad {
+
+constexpr int kBlock = 256;
+constexpr int kUnroll = 4;
+
+// ---------------------------------------------------------------- storage types
+
+struct StoreF32 {
+    using elem = float;
+    static constexpr int kVec = 4;             // elements per 16-byte packet
+    static __device__ __forceinline__ void unpack(const uint4& p, float (&v)[4])
+    {
+        v[0] = __uint_as_float(p.x); v[1] = __uint_as_float(p.y);
+        v[2] = __uint_as_float(p.z); v[3] = __uint_as_float(p.w);
+    }
+    static __device__ __forceinline__ uint4 pack(const float (&v)[4])
+    {
+        return make_uint4(__float_as_uint(v[0]), __float_as_uint(v[1]), __float_as_uint(v[2]), __float_as_uint(v[3]));
+    }
+    static __device__ __forceinline__ float load1(const elem* p) { return *p; }
+    static __device__ __forceinline__ void store1(elem* p, float v) { *p = v; }
+};
+
+struct StoreBF16 {
+    using elem = __nv_bfloat16;
+    static constexpr int kVec = 8;
+    // a bf16 is the upper half of an fp32: widening is a shift or a mask
+    static __device__ __forceinline__ void unpack(const uint4& p, float (&v)[8])
+    {
+        const uint32_t w[4] = {p.x, p.y, p.z, p.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            v[2 * i] = __uint_as_float(w[i] << 16);
+            v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+        }
+    }
+    static __device__ __forceinline__ uint32_t pack2(float lo, float hi)
+    {
+        __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);   // cvt.rn.bf16x2.f32: round to nearest even
+        return *reinterpret_cast<uint32_t*>(&h);
+    }
+    static __device__ __forceinline__ uint4 pack(const float (&v)[8])
+    {
+        return make_uint4(pack2(v[0], v[1]), pack2(v[2], v[3]), pack2(v[4], v[5]), pack2(v[6], v[7]));
+    }
+    static __device__ __forceinline__ float load1(const elem* p) { return __bfloat162float(*p); }
+    static __device__ __forceinline__ void store1(elem* p, float v) { *p = __float2bfloat16_rn(v); }
+};
+
+struct StoreF16 {
+    using elem = __half;
+    static constexpr int kVec = 8;
+    static __device__ __forceinline__ void unpack(const uint4& p, float (&v)[8])
+    {
+        const uint32_t w[4] = {p.x, p.y, p.z, p.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            float2 f = __half22float2(*reinterpret_cast<const __half2*>(&w[i]));
+            v[2 * i] = f.x;
+            v[2 * i + 1] = f.y;
+        }
+    }
+    static __device__ __forceinline__ uint32_t pack2(float lo, float hi)
+    {
+        __half2 h = __floats2half2_rn(lo, hi);              // cvt.rn.f16x2.f32
+        return *reinterpret_cast<uint32_t*>(&h);
+    }
+    static __device__ __forceinline__ uint4 pack(const float (&v)[8])
+    {
+        return make_uint4(pack2(v[0], v[1]), pack2(v[2], v[3]), pack2(v[4], v[5]), pack2(v[6], v[7]));
+    }
+    static __device__ __forceinline__ float load1(const elem* p) { return __half2float(*p); }
+    static __device__ __forceinline__ void store1(elem* p, float v) { *p = __float2half_rn(v); }
+};
+
+// ---------------------------------------------------------------- memory access with cache hints
+
+// Inputs are read once: streaming (evict-first) loads.
+__device__ __forceinline__ uint4 load_packet(const uint4* p) { return __ldcs(p); }
+
+// Output slot `keep`: true for a tensor the next kernel reads at once (y, grad_in),
+// false for one that is read much later or never by this stream (the saved f').
+template <bool kKeep> __device__ __forceinline__ void store_packet(uint4* p, const uint4& v)
+{
+    if (kKeep) *p = v;
+    else __stcs(p, v);
+}
+
+// ---------------------------------------------------------------- kernel
+
+template <int NIN, int NOUT> struct StreamArgs {
+    const void* in[NIN];
+    void* out[NOUT];
+    size_t n;          // elements
+    size_t head;       // elements before the first 16-byte boundary (same for every tensor)
+    size_t packets;    // whole packets after the head
+};
+
+// Op: struct with
+//   static constexpr int kIn, kOut;  static constexpr bool kKeep[kOut];
+//   static __device__ void apply(const float (&in)[kIn], float (&out)[kOut]);
+template <class S, class Op>
+__device__ __forceinline__ void scalar_element(const StreamArgs<Op::kIn, Op::kOut>& a, size_t i)
+{
+    using E = typename S::elem;
+    float in[Op::kIn], out[Op::kOut];
+#pragma unroll
+    for (int k = 0; k < Op::kIn; ++k) in[k] = S::load1(static_cast<const E*>(a.in[k]) + i);
+    Op::apply(in, out);
+#pragma unroll
+    for (int k = 0; k < Op::kOut; ++k) S::store1(static_cast<E*>(a.out[k]) + i, out[k]);
+}
+
+template <class S, class Op>
+__device__ __forceinline__ void packet_compute_store(const StreamArgs<Op::kIn, Op::kOut>& a, size_t pk,
+                                                     const uint4 (&raw)[Op::kIn])
+{
+    constexpr int V = S::kVec;
+    float vin[Op::kIn][V];
+    float vout[Op::kOut][V];
+#pragma unroll
+    for (int k = 0; k < Op::kIn; ++k) S::unpack(raw[k], vin[k]);
+#pragma unroll
+    for (int e = 0; e < V; ++e) {
+        float in[Op::kIn], out[Op::kOut];
+#pragma unroll
+        for (int k = 0; k < Op::kIn; ++k) in[k] = vin[k][e];
+        Op::apply(in, out);
+#pragma unroll
+        for (int k = 0; k < Op::kOut; ++k) vout[k][e] = out[k];
+    }
+    const size_t byte_off = a.head * sizeof(typename S::elem);
+#pragma unroll
+    for (int k = 0; k < Op::kOut; ++k) {
+        uint4* dst = reinterpret_cast<uint4*>(static_cast<char*>(a.out[k]) + byte_off) + pk;
+        uint4 v = S::pack(vout[k]);
+        if (Op::keep(k)) store_packet<true>(dst, v);
+        else store_packet<false>(dst, v);
+    }
+}
+
+template <class S, class Op>
+__global__ void __launch_bounds__(kBlock) stream_kernel(const StreamArgs<Op::kIn, Op::kOut> a)
+{
+    constexpr int V = S::kVec;
+    const size_t byte_off = a.head * sizeof(typename S::elem);
+    const size_t tile_packets = size_t(kBlock) * kUnroll;
+    const size_t n_tiles = (a.packets + tile_packets - 1) / tile_packets;
+
+    for (size_t tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
+        const size_t base = tile * tile_packets + threadIdx.x;
+        uint4 raw[kUnroll][Op::kIn];
+        if (base + size_t(kUnroll - 1) * kBlock < a.packets) {          // whole tile: no predicates
+#pragma unroll
+            for (int u = 0; u < kUnroll; ++u)
+#pragma unroll
+                for (int k = 0; k < Op::kIn; ++k)
+                    raw[u][k] = load_packet(reinterpret_cast<const uint4*>(static_cast<const char*>(a.in[k]) + byte_off) +
+                                            base + size_t(u) * kBlock);
+#pragma unroll
+            for (int u = 0; u < kUnroll; ++u) packet_compute_store<S, Op>(a, base + size_t(u) * kBlock, raw[u]);
+        } else {
+#pragma unroll
+            for (int u = 0; u < kUnroll; ++u) {
+                const size_t pk = base + size_t(u) * kBlock;
+                if (pk < a.packets) {
+#pragma unroll
+                    for (int k = 0; k < Op::kIn; ++k)
+                        raw[u][k] = load_packet(reinterpret_cast<const uint4*>(static_cast<const char*>(a.in[k]) + byte_off) + pk);
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < kUnroll; ++u) {
+                const size_t pk = base + size_t(u) * kBlock;
+                if (pk < a.packets) packet_compute_store<S, Op>(a, pk, raw[u]);
+            }
+        }
+    }
+
+    // ragged ends: at most V-1 elements before the first packet and after the last
+    if (blockIdx.x == 0) {
+        const size_t tail_begin = a.head + a.packets * V;
+        const size_t n_edge = a.head + (a.n - tail_begin);
+        for (size_t j = threadIdx.x; j < n_edge; j += kBlock) {
+            const size_t i = j < a.head ? j : tail_begin + (j - a.head);
+            scalar_element<S, Op>(a, i);
+        }
+    }
+}
+
+// Every element one by one: taken when the tensors do not share one offset
+// modulo 16 bytes, so that no common packet grid exists.
+template <class S, class Op>
+__global__ void __launch_bounds__(kBlock) scalar_kernel(const StreamArgs<Op::kIn, Op::kOut> a)
+{
+    const size_t stride = size_t(gridDim.x) * kBlock;
+    for (size_t i = size_t(blockIdx.x) * kBlock + threadIdx.x; i < a.n; i += stride) scalar_element<S, Op>(a, i);
+}
+
+// ---------------------------------------------------------------- launch
+
+struct DeviceInfo { int sm_count; };
+
+inline cudaError_t device_info(DeviceInfo* out)
+{
+    static thread_local int cached_dev = -1;
+    static thread_local DeviceInfo cached;
+    int dev;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev != cached_dev) {
+        e = cudaDeviceGetAttribute(&cached.sm_count, cudaDevAttrMultiProcessorCount, dev);
+        if (e != cudaSuccess) return e;
+        cached_dev = dev;
+    }
+    *out = cached;
+    return cudaSuccess;
+}
+
+template <class S, class Op>
+cudaError_t launch_stream(const void* const* in, void* const* out, size_t n, cudaStream_t st)
+{
+    if (n == 0) return cudaSuccess;
+    StreamArgs<Op::kIn, Op::kOut> a;
+    uintptr_t mis = 0;
+    bool congruent = true;
+    for (int k = 0; k < Op::kIn; ++k) {
+        a.in[k] = in[k];
+        uintptr_t m = reinterpret_cast<uintptr_t>(in[k]) & 15u;
+        if (k == 0) mis = m;
+        congruent = congruent && (m == mis);
+    }
+    for (int k = 0; k < Op::kOut; ++k) {
+        a.out[k] = out[k];
+        congruent = congruent && ((reinterpret_cast<uintptr_t>(out[k]) & 15u) == mis);
+    }
+    a.n = n;
+    DeviceInfo di;
+    cudaError_t e = device_info(&di);
+    if (e != cudaSuccess) return e;
+
+    static thread_local int occ_stream = 0, occ_scalar = 0;   // per instantiation
+    if (!congruent) {
+        if (occ_scalar == 0) {
+            e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ_scalar, scalar_kernel<S, Op>, kBlock, 0);
+            if (e != cudaSuccess) return e;
+        }
+        a.head = 0;
+        a.packets = 0;
+        size_t blocks = (n + kBlock - 1) / kBlock;
+        size_t cap = size_t(di.sm_count) * occ_scalar;
+        scalar_kernel<S, Op><<<(unsigned)(blocks < cap ? blocks : cap), kBlock, 0, st>>>(a);
+        return cudaPeekAtLastError();
+    }
+    constexpr size_t esz = sizeof(typename S::elem);
+    size_t head = ((16u - mis) & 15u) / esz;
+    if (head > n) head = n;
+    a.head = head;
+    a.packets = (n - head) / S::kVec;
+    if (occ_stream == 0) {
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ_stream, stream_kernel<S, Op>, kBlock, 0);
+        if (e != cudaSuccess) return e;
+    }
+    const size_t tile_packets = size_t(kBlock) * kUnroll;
+    size_t tiles = (a.packets + tile_packets - 1) / tile_packets;
+    if (tiles == 0) tiles = 1;                                  // edges only
+    size_t cap = size_t(di.sm_count) * occ_stream;
+    stream_kernel<S, Op><<<(unsigned)(tiles < cap ? tiles : cap), kBlock, 0, st>>>(a);
+    return cudaPeekAtLastError();
+}
+
+}  // namespace nfad

@@ -1,0 +1,114 @@
+"""Shared parity checks: CUDA results against the fp64 oracle on the same arrays.
+
+Tolerances (stated once, used by every GPU test):
+  fp32 y      : |got - o| <= 4 ulp32(o)                      (normal-range o)
+  fp32 f'     : x >= 0: |got - o| <= 4 ulp32(o)
+                x <  0: |got - o| <= 4 ulp32(T), T = |h| + |x h'|, because f' = h + x h'
+                        is there a difference of two fp32-evaluated terms and changes sign;
+                        no fp32-internal evaluation can hold 4 ulp of a result that is ~0
+  fp32, |o| < 2^-126 (subnormal result): |got - o| <= 64 * 2^-149
+  bf16 / fp16 : |ord(got) - ord(RN(o))| <= 1, RN = one rounding from fp64
+  backward    : bit-equal to RN(fp64(g) * fp64(f'_saved)), f'_saved being the GPU's own tensor
+"""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+import oracle
+import ulp
+from paper_2209_10778_b200 import binding as nfad
+from paper_2209_10778_b200 import workloads as W
+
+FP32_ULPS = 4.0
+SUBNORMAL_SLACK = 64 * 2.0 ** -149
+MIN_NORMAL = 2.0 ** -126
+
+
+def gpu_forward(kind: str, x: torch.Tensor):
+    y = torch.empty_like(x)
+    d = torch.empty_like(x)
+    nfad.nfad_act_forward(kind, x, y, d)
+    return y, d
+
+
+def gpu_backward(kind: str, g: torch.Tensor, d: torch.Tensor):
+    gin = torch.empty_like(g)
+    nfad.nfad_act_backward(kind, g, d, gin)
+    return gin
+
+
+def _fail_report(name, bad, x, got, want, err):
+    idx = np.flatnonzero(bad)
+    worst = idx[np.argmax(err[idx])]
+    return (f"{name}: {idx.size} of {bad.size} elements out of tolerance; worst at i={worst}: x={x[worst]!r} "
+            f"got={got[worst]!r} oracle={want[worst]!r} err={err[worst]:.3f}")
+
+
+def check_forward_fp32(kind: str, x_raw: np.ndarray, y: np.ndarray, d: np.ndarray, stats: dict | None = None):
+    f, fp, cond = oracle.forward(kind, "f32", x_raw, want_cond=True)
+    xd = x_raw.astype(np.float64)
+    # value
+    ey = ulp.err_strict32(y, f)
+    sub = np.abs(f) < MIN_NORMAL
+    bad = np.where(sub, np.abs(y.astype(np.float64) - f) > SUBNORMAL_SLACK, ey > FP32_ULPS) | ~np.isfinite(y)
+    assert not bad.any(), _fail_report(f"{kind} fp32 y", bad, x_raw, y, f, ey)
+    # derivative
+    es = ulp.err_strict32(d, fp)
+    ec = ulp.err_scaled32(d, fp, cond)
+    gate = np.where(xd >= 0, es, ec)
+    subd = np.abs(fp) < MIN_NORMAL
+    # (a subnormal f' next to its sign change still has normal-sized addends: scaled gate)
+    tail = subd & (cond < 2.0 ** -100)
+    badd = np.where(tail, np.abs(d.astype(np.float64) - fp) > SUBNORMAL_SLACK, gate > FP32_ULPS) | ~np.isfinite(d)
+    assert not badd.any(), _fail_report(f"{kind} fp32 f'", badd, x_raw, d, fp, gate)
+    if stats is not None:
+        neg = xd < 0
+        stats.update(
+            y_max_ulp=float(ey[~sub].max(initial=0.0)),
+            d_gate_max=float(gate[~subd].max(initial=0.0)),
+            d_strict_max=float(es[~subd].max(initial=0.0)),
+            d_strict_p999=float(np.quantile(es[neg & ~subd], 0.999)) if (neg & ~subd).any() else 0.0,
+            d_only_scaled=int(((es > FP32_ULPS) & ~subd).sum()),
+        )
+
+
+def check_forward_16(kind: str, dtype: str, x_raw: np.ndarray, y_bits: np.ndarray, d_bits: np.ndarray,
+                     stats: dict | None = None):
+    f, fp = oracle.forward(kind, dtype, x_raw)
+    want_y = oracle.round_to(dtype, f)
+    want_d = oracle.round_to(dtype, fp)
+    dy = ulp.ulp_distance16(y_bits, want_y)
+    dd = ulp.ulp_distance16(d_bits, want_d)
+    xw = oracle.widen(dtype, x_raw)
+    bad = (dy > 1) | ulp.is_nan16(y_bits, dtype)
+    assert not bad.any(), _fail_report(f"{kind} {dtype} y", bad, xw, oracle.widen(dtype, y_bits), f, dy.astype(np.float64))
+    badd = (dd > 1) | ulp.is_nan16(d_bits, dtype)
+    assert not badd.any(), _fail_report(f"{kind} {dtype} f'", badd, xw, oracle.widen(dtype, d_bits), fp, dd.astype(np.float64))
+    if stats is not None:
+        stats.update(y_off_by_one=int((dy == 1).sum()), d_off_by_one=int((dd == 1).sum()))
+
+
+def check_backward(dtype: str, g_raw: np.ndarray, d_raw: np.ndarray, gin_raw: np.ndarray):
+    want = oracle.backward(dtype, g_raw, d_raw)
+    same = ulp.same_bits_or_both_nan(gin_raw, want, dtype)
+    if not same.all():
+        i = int(np.flatnonzero(~same)[0])
+        raise AssertionError(f"backward {dtype}: {int((~same).sum())} mismatches; first at i={i}: "
+                             f"g={oracle.widen(dtype, g_raw[i:i+1])[0]!r} f'={oracle.widen(dtype, d_raw[i:i+1])[0]!r} "
+                             f"got={oracle.widen(dtype, gin_raw[i:i+1])[0]!r} want={oracle.widen(dtype, want[i:i+1])[0]!r}")
+
+
+def full_check(kind: str, dtype: str, x: torch.Tensor, g: torch.Tensor, stats: dict | None = None):
+    """Forward + backward through the C-ABI on CUDA tensors x, g; compare everything with the oracle."""
+    y, d = gpu_forward(kind, x)
+    gin = gpu_backward(kind, g, d)
+    torch.cuda.synchronize()
+    x_raw, g_raw = W.raw_numpy(x), W.raw_numpy(g)
+    y_raw, d_raw, gin_raw = W.raw_numpy(y), W.raw_numpy(d), W.raw_numpy(gin)
+    if dtype == "f32":
+        check_forward_fp32(kind, x_raw, y_raw, d_raw, stats)
+    else:
+        check_forward_16(kind, dtype, x_raw, y_raw, d_raw, stats)
+    check_backward(dtype, g_raw, d_raw, gin_raw)
+    return y, d, gin

@@ -1,0 +1,80 @@
+"""Host-side checks of the C-ABI library that need no GPU: it loads, exports exactly
+the symbols the header declares, and validates arguments before touching CUDA."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from paper_2209_10778_b200 import binding, build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    build.build_library()
+    return binding.load()
+
+
+def _declared_symbols():
+    text = open(os.path.join(ROOT, "include", "nfad.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"NFAD_API\s+[\w\s\*]+?\b(nfad_\w+)\s*\(", text)))
+
+
+def test_header_and_binding_agree_on_the_exports():
+    assert _declared_symbols() == sorted(binding.EXPORTS)
+
+
+def test_library_exports_every_declared_symbol(lib):
+    for name in _declared_symbols():
+        assert hasattr(lib, name), name
+
+
+def test_no_other_nfad_symbols_are_exported(lib):
+    import subprocess
+    out = subprocess.run(["nm", "-D", "--defined-only", binding.LIB_PATH], capture_output=True, text=True).stdout
+    exported = sorted(l.split()[-1] for l in out.splitlines() if " T " in l)
+    assert exported == _declared_symbols()
+
+
+def test_version_and_status_strings(lib):
+    assert re.fullmatch(r"\d+\.\d+\.\d+", binding.nfad_version())
+    assert binding.nfad_status_string(0) == "ok"
+    assert len({binding.nfad_status_string(i) for i in range(9)}) == 9
+
+
+def test_validation_needs_no_device(lib):
+    fake = ctypes.c_void_p(0x1000)
+    assert lib.nfad_act_forward(4, 0, fake, fake, fake, 8, None) == 1        # kind
+    assert lib.nfad_act_forward(-1, 0, fake, fake, fake, 8, None) == 1
+    assert lib.nfad_act_forward(0, 3, fake, fake, fake, 8, None) == 2        # dtype
+    assert lib.nfad_act_forward(0, 0, None, fake, fake, 8, None) == 3        # null
+    assert lib.nfad_act_backward(0, 0, fake, None, fake, 8, None) == 3
+    assert lib.nfad_act_forward(0, 0, fake, ctypes.c_void_p(0x2000), ctypes.c_void_p(0x2010), 8, None) == 4   # y, dfdx overlap
+    assert lib.nfad_act_forward_infer(0, 0, fake, ctypes.c_void_p(0x1004), 8, None) == 4                      # partial overlap
+    assert lib.nfad_act_forward(0, 0, ctypes.c_void_p(0x1002), fake, ctypes.c_void_p(0x3000), 8, None) == 6   # alignment
+    assert lib.nfad_act_forward(0, 1, ctypes.c_void_p(0x1001), fake, ctypes.c_void_p(0x3000), 8, None) == 6
+    # n == 0 is valid with any pointers and launches nothing
+    assert lib.nfad_act_forward(0, 0, None, None, None, 0, None) == 0
+    assert lib.nfad_act_backward(3, 2, None, None, None, 0, None) == 0
+    assert lib.nfad_cmp_recompute_backward(0, 0, fake, fake, fake, 0, fake, 8, None) == 7                    # scratch too small
+
+
+def test_saved_bytes_and_scratch_size(lib):
+    assert lib.nfad_saved_bytes_per_element(2, 1, 0) == 2
+    assert lib.nfad_saved_bytes_per_element(2, 1, 3) == 4
+    assert lib.nfad_saved_bytes_per_element(1, 0, 3) == 16
+    assert lib.nfad_saved_bytes_per_element(0, 0, 9) == -8
+    assert lib.nfad_saved_bytes_per_element(7, 0, 0) == -1
+    assert lib.nfad_cmp_recompute_scratch_bytes(0, 1, 1000) == 2000
+    assert lib.nfad_cmp_recompute_scratch_bytes(0, 0, 3) == 16
+    assert lib.nfad_cmp_recompute_scratch_bytes(9, 0, 3) == 0
+
+
+def test_binding_refuses_cpu_tensors():
+    import torch
+    x = torch.zeros(8)
+    with pytest.raises(TypeError):
+        binding.nfad_act_forward("swish", x, x.clone(), x.clone())

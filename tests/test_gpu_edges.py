@@ -1,0 +1,172 @@
+"""GPU edge cases: sizes around packet and tile boundaries, unaligned and mutually
+misaligned pointers, in-place use, guard bands around every output, error returns,
+and the two comparator layouts."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import parity
+import ulp
+from paper_2209_10778_b200 import binding as nfad
+from paper_2209_10778_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+KINDS = list(W.KINDS)
+SIZES = [0, 1, 2, 3, 7, 8, 9, 15, 16, 17, 255, 256, 257, 1023, 1025, 4095, 4096, 4097, 8191, 8193, 32767, 32769, 65535, 65537]
+
+
+def _guarded(n, td, pad=64, fill=7.0):
+    """A tensor of n elements inside a larger buffer whose margins must stay untouched."""
+    buf = torch.full((n + 2 * pad,), fill, dtype=td, device=DEV)
+    return buf, buf[pad:pad + n]
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16", "f16"])
+def test_sizes_and_guard_bands(dtype):
+    td = W.TORCH_DTYPES[dtype]
+    kind = "gelu_tanh"
+    for n in SIZES:
+        x = W.draw("normal", max(n, 1), dtype, n, DEV)[:n].contiguous()
+        g = W.normal(max(n, 1), dtype, n + 1, 1.0, DEV)[:n].contiguous()
+        yb, y = _guarded(n, td)
+        db, d = _guarded(n, td)
+        gb, gin = _guarded(n, td)
+        nfad.nfad_act_forward(kind, x, y, d)
+        nfad.nfad_act_backward(kind, g, d, gin)
+        torch.cuda.synchronize()
+        for b in (yb, db, gb):
+            assert (b[:64] == 7.0).all() and (b[64 + n:] == 7.0).all(), f"guard band touched at n={n}"
+        if n:
+            xr = W.raw_numpy(x)
+            if dtype == "f32":
+                parity.check_forward_fp32(kind, xr, W.raw_numpy(y), W.raw_numpy(d))
+            else:
+                parity.check_forward_16(kind, dtype, xr, W.raw_numpy(y), W.raw_numpy(d))
+            parity.check_backward(dtype, W.raw_numpy(g), W.raw_numpy(d), W.raw_numpy(gin))
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16", "f16"])
+def test_unaligned_and_misaligned_pointers_give_identical_bits(dtype):
+    td = W.TORCH_DTYPES[dtype]
+    n = 20011
+    kind = "mish"
+    x0 = W.draw("mix", n, dtype, 11, DEV)
+    y0, d0 = parity.gpu_forward(kind, x0)
+    per16 = 16 // x0.element_size()
+    for ox, oy, od in [(1, 1, 1), (3, 3, 3), (per16 - 1, per16 - 1, per16 - 1), (0, 1, 2), (1, 0, 0), (2, 2, 1)]:
+        xb = torch.zeros(n + 16, dtype=td, device=DEV)
+        yb = torch.full((n + 16,), 7.0, dtype=td, device=DEV)
+        db = torch.full((n + 16,), 7.0, dtype=td, device=DEV)
+        xb[ox:ox + n] = x0
+        nfad.nfad_act_forward(kind, xb[ox:ox + n], yb[oy:oy + n], db[od:od + n])
+        torch.cuda.synchronize()
+        assert np.array_equal(W.raw_numpy(yb[oy:oy + n]), W.raw_numpy(y0)), (ox, oy, od)
+        assert np.array_equal(W.raw_numpy(db[od:od + n]), W.raw_numpy(d0)), (ox, oy, od)
+        assert (yb[:oy] == 7.0).all() and (yb[oy + n:] == 7.0).all()
+        assert (db[:od] == 7.0).all() and (db[od + n:] == 7.0).all()
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_in_place(dtype):
+    n = 50001
+    kind = "swish"
+    x = W.draw("normal", n, dtype, 21, DEV)
+    g = W.normal(n, dtype, 22, 1.0, DEV)
+    y0, d0 = parity.gpu_forward(kind, x)
+    gin0 = parity.gpu_backward(kind, g, d0)
+    # y in place of x
+    xa = x.clone(); da = torch.empty_like(x)
+    nfad.nfad_act_forward(kind, xa, xa, da)
+    # dfdx in place of x
+    xb = x.clone(); yb = torch.empty_like(x)
+    nfad.nfad_act_forward(kind, xb, yb, xb)
+    # grad_in in place of grad_out, and of dfdx
+    ga = g.clone(); nfad.nfad_act_backward(kind, ga, d0, ga)
+    dc = d0.clone(); nfad.nfad_act_backward(kind, g, dc, dc)
+    torch.cuda.synchronize()
+    assert torch.equal(xa, y0) and torch.equal(da, d0)
+    assert torch.equal(yb, y0) and torch.equal(xb, d0)
+    assert torch.equal(ga, gin0) and torch.equal(dc, gin0)
+
+
+def test_error_returns_on_device_pointers():
+    x = torch.zeros(1024, device=DEV)
+    y = torch.zeros(1024, device=DEV)
+    with pytest.raises(nfad.NfadError) as e:
+        nfad.nfad_act_forward("swish", x, y, y)            # two outputs overlap
+    assert e.value.status == 4
+    with pytest.raises(nfad.NfadError) as e:
+        nfad.nfad_act_forward("swish", x[:512], x[256:768], y[:512])   # partial overlap of input and output
+    assert e.value.status == 4
+    with pytest.raises(nfad.NfadError) as e:
+        nfad.nfad_act_forward(11, x, y, torch.zeros(1024, device=DEV))
+    assert e.value.status == 1
+    torch.cuda.synchronize()
+
+
+def _conv_tolerance_ok(dtype, gin_raw, g_raw, x_raw, kind):
+    """Conventional backward multiplies g by an fp32 f'(x) that is never rounded to the storage
+    type: |gin - g f'| <= |g| * 4 ulp32(T) plus one rounding of the product to the storage type."""
+    f, fp, cond = oracle.forward(kind, dtype, x_raw, want_cond=True)
+    g = oracle.widen(dtype, g_raw)
+    want = g * fp
+    got = oracle.widen(dtype, gin_raw)
+    tol32 = np.abs(g) * 4 * ulp.ulp32(cond)
+    if dtype == "f32":
+        tol = tol32 + 0.5 * ulp.ulp32(want) * 1.0001
+    else:
+        rn = oracle.widen(dtype, oracle.round_to(dtype, want))
+        up = oracle.widen(dtype, oracle.round_to(dtype, want + tol32))
+        lo = oracle.widen(dtype, oracle.round_to(dtype, want - tol32))
+        return (got >= np.minimum(lo, rn)) & (got <= np.maximum(up, rn))
+    return np.abs(got - want) <= tol + 64 * 2.0 ** -149
+
+
+@pytest.mark.parametrize("kind", KINDS)
+@pytest.mark.parametrize("dtype", ["f32", "bf16", "f16"])
+def test_conventional_comparator(kind, dtype):
+    n = (1 << 16) + 5
+    x = W.draw("normal", n, dtype, 31, DEV)
+    g = W.normal(n, dtype, 32, 1.0, DEV)
+    gin = torch.empty_like(g)
+    nfad.nfad_cmp_conv_backward(kind, g, x, gin)
+    torch.cuda.synchronize()
+    ok = _conv_tolerance_ok(dtype, W.raw_numpy(gin), W.raw_numpy(g), W.raw_numpy(x), kind)
+    assert ok.all(), f"{(~ok).sum()} of {n} outside tolerance"
+
+
+@pytest.mark.parametrize("kind", KINDS)
+@pytest.mark.parametrize("dtype", ["f32", "bf16", "f16"])
+def test_recompute_comparator(kind, dtype):
+    # operator-by-operator rules through a stored intermediate: the tolerance is the one that
+    # arithmetic has -- an absolute error of a few storage-type ulps of the gate, times |g| (1 + |x|)
+    n = (1 << 16) + 5
+    x = W.draw("normal", n, dtype, 41, DEV)
+    g = W.normal(n, dtype, 42, 1.0, DEV)
+    gin = torch.empty_like(g)
+    nbytes = nfad.nfad_cmp_recompute_scratch_bytes(kind, dtype, n)
+    assert nbytes >= n * x.element_size()
+    scratch = torch.empty(nbytes, dtype=torch.uint8, device=DEV)
+    nfad.nfad_cmp_recompute_backward(kind, g, x, scratch, gin)
+    torch.cuda.synchronize()
+    f, fp = oracle.forward(kind, dtype, W.raw_numpy(x))
+    gw, xw = oracle.widen(dtype, W.raw_numpy(g)), oracle.widen(dtype, W.raw_numpy(x))
+    got = oracle.widen(dtype, W.raw_numpy(gin))
+    eps = {"f32": 2.0 ** -23, "bf16": 2.0 ** -8, "f16": 2.0 ** -11}[dtype]
+    tol = np.abs(gw) * eps * 4 * (1 + 2 * np.abs(xw)) + eps * np.abs(gw * fp)
+    assert (np.abs(got - gw * fp) <= tol).all()
+    with pytest.raises(nfad.NfadError) as e:
+        nfad.nfad_cmp_recompute_backward(kind, g, x, scratch[:16], gin)
+    assert e.value.status == 7
+
+
+def test_saved_bytes_per_element_table():
+    for dtype, s in (("f32", 4), ("bf16", 2), ("f16", 2)):
+        for kind in KINDS:
+            assert nfad.nfad_saved_bytes_per_element(kind, dtype, "nested") == s
+            assert nfad.nfad_saved_bytes_per_element(kind, dtype, "conventional") == s
+            assert nfad.nfad_saved_bytes_per_element(kind, dtype, "recompute") == s
+            assert nfad.nfad_saved_bytes_per_element(kind, dtype, "op_by_op") >= 2 * s
+        assert nfad.nfad_saved_bytes_per_element("swish", dtype, "op_by_op") == 2 * s   # x and sigmoid(x)
