@@ -1,8 +1,8 @@
 // nfad_dual.cuh -- the device-side dual-number algebra of nested Forward-AD.
 //
 // A dual number carries a value v and a tangent t = dv/dx.  Every primitive
-// computes its value and its derivative TOGETHER (Section II-C, approach 3:
-// "v1' = v1(1-v1) is calculated when v1 is executed"), sharing the one
+// computes its value and its derivative TOGETHER (Section II-C, approach 3: the
+// derivative of a node is calculated when the node is executed), sharing the one
 // exponential that both need; a unary primitive applies the chain rule
 // t_out = prim'(v) * t_in, and the product of two duals of the same source
 // applies the product rule of Eq. 3.  The seed is x' = 1 (Section II-D), held
@@ -14,17 +14,24 @@
 // the closed symbolic forms tanh / sigmoid / softplus that frameworks ship as
 // single operators):
 //     dual_add  dual_mul  dual_scale  dual_add_const
-//     dual_exp  dual_log1p  dual_tanh  dual_erf  dual_softplus  dual_sigmoid
+//     dual_tanh  dual_softplus  dual_sigmoid
 // and two "binary with a constant, hence unary" fusions that keep the tails
 // free of cancellation:
 //     dual_half_one_plus_tanh(u) = (1 + tanh u)/2 = sigmoid(2u)
 //     dual_half_one_plus_erf(z)  = (1 + erf z)/2  = erfc(-z)/2
 //
-// Under the Full policy (fp32 storage) a value is an unevaluated sum v + vl so
-// that (a) arguments of exponentials keep the bits that |arg| would otherwise
-// amplify and (b) a result of the form 1 - small is held as (1, -small) and
-// rounded once, at the store.  Under the Fast policy (16-bit storage) a value is
-// one float.
+// Policies.  Fast (16-bit storage): a value and a tangent are one float each.
+// Full (fp32 storage): both are unevaluated sums hi + lo.  That keeps (a) the
+// bits of an exponential's argument that |arg| would amplify, (b) a result of
+// the form 1 - small as the pair (1, -small), and (c) the two addends of the
+// product rule exact enough that their cancellation for x < 0 costs nothing
+// beyond the accuracy of the exponential itself; everything is rounded once, at
+// the store.
+//
+// Gates.  sigmoid, (1+tanh)/2, (1+erf)/2 and tanh(softplus) all behave like
+// exp(-|v|) on their small side.  Under Full they return a `Gate`: a dual whose
+// value and tangent share a factor 2^kexp that is applied last (it is exact),
+// so that nothing on the way is rounded in the subnormal range.
 #pragma once
 
 #include "nfad_numerics.cuh"
@@ -36,61 +43,71 @@ struct Seed { float x; };
 
 template <class P> struct Dual;
 template <> struct Dual<Fast> { float v, t; };
-template <> struct Dual<Full> { float v, vl, t; };
+template <> struct Dual<Full> { F2 v, t; };
+
+template <class P> struct Gate;
+template <> struct Gate<Fast> { float v, t; };
+template <> struct Gate<Full> { F2 v, t; int kexp; };     // 2^kexp (v, t)
 
 // A constant known to more than fp32 precision.
 struct Const2 { float h, l; };
 
 NFAD_DEV float dual_value(const Dual<Fast>& a) { return a.v; }
-NFAD_DEV float dual_value(const Dual<Full>& a) { return a.v + a.vl; }   // the one rounding
+NFAD_DEV float dual_tangent(const Dual<Fast>& a) { return a.t; }
+NFAD_DEV float dual_value(const Gate<Fast>& a) { return a.v; }
+NFAD_DEV float dual_tangent(const Gate<Fast>& a) { return a.t; }
+NFAD_DEV float dual_value(const Dual<Full>& a) { return f2_value(a.v); }       // the one rounding
+NFAD_DEV float dual_tangent(const Dual<Full>& a) { return f2_value(a.t); }
+NFAD_DEV float dual_value(const Gate<Full>& a) { return scale_pow2(f2_value(a.v), a.kexp); }
+NFAD_DEV float dual_tangent(const Gate<Full>& a) { return scale_pow2(f2_value(a.t), a.kexp); }
+
+// A gate as an ordinary dual (for further generic composition).
+NFAD_DEV Dual<Fast> as_dual(const Gate<Fast>& a) { return {a.v, a.t}; }
+NFAD_DEV Dual<Full> as_dual(const Gate<Full>& a)
+{
+    float s = pow2_clamped(a.kexp);
+    return {{a.v.h * s, a.v.l * s}, {a.t.h * s, a.t.l * s}};
+}
 
 // ----------------------------------------------------------------- add, scale (linear)
 
 NFAD_DEV Dual<Fast> dual_add(const Dual<Fast>& a, const Dual<Fast>& b) { return {a.v + b.v, a.t + b.t}; }
-NFAD_DEV Dual<Full> dual_add(const Dual<Full>& a, const Dual<Full>& b)
-{
-    F2 s = two_sum(a.v, b.v);
-    return {s.h, s.l + (a.vl + b.vl), a.t + b.t};
-}
+NFAD_DEV Dual<Full> dual_add(const Dual<Full>& a, const Dual<Full>& b) { return {f2_add(a.v, b.v), f2_add(a.t, b.t)}; }
 
 // c + a (binary with one constant input: unary, tangent unchanged)
 NFAD_DEV Dual<Fast> dual_add_const(float c, const Dual<Fast>& a) { return {c + a.v, a.t}; }
 NFAD_DEV Dual<Full> dual_add_const(float c, const Dual<Full>& a)
 {
-    F2 s = two_sum(c, a.v);
-    return {s.h, s.l + a.vl, a.t};
+    F2 s = two_sum(c, a.v.h);
+    s.l += a.v.l;
+    return {s, a.t};
 }
 
 // c * a
 NFAD_DEV Dual<Fast> dual_scale(Const2 c, const Dual<Fast>& a) { return {c.h * a.v, c.h * a.t}; }
 NFAD_DEV Dual<Full> dual_scale(Const2 c, const Dual<Full>& a)
 {
-    F2 p = two_prod(c.h, a.v);
-    return {p.h, fmaf(c.h, a.vl, fmaf(c.l, a.v, p.l)), c.h * a.t};
+    return {f2_mul(a.v, F2{c.h, c.l}), f2_mul(a.t, F2{c.h, c.l})};
 }
 // (a seed does not say which policy its result takes: the caller passes it as a tag)
 NFAD_DEV Dual<Fast> dual_scale(Fast, Const2 c, const Seed& a) { return {c.h * a.x, c.h}; }
-NFAD_DEV Dual<Full> dual_scale(Full, Const2 c, const Seed& a)
-{
-    F2 p = two_prod(c.h, a.x);
-    return {p.h, fmaf(c.l, a.x, p.l), c.h};
-}
+NFAD_DEV Dual<Full> dual_scale(Full, Const2 c, const Seed& a) { return {f2_mul(F2{c.h, c.l}, a.x), {c.h, c.l}}; }
 
 // ----------------------------------------------------------------- mul (product rule, Eq. 3)
 
 NFAD_DEV Dual<Fast> dual_mul(Fast, const Seed& a, const Seed& b) { return {a.x * b.x, a.x + b.x}; }
-NFAD_DEV Dual<Full> dual_mul(Full, const Seed& a, const Seed& b)
-{
-    F2 p = two_prod(a.x, b.x);
-    return {p.h, p.l, a.x + b.x};
-}
+NFAD_DEV Dual<Full> dual_mul(Full, const Seed& a, const Seed& b) { return {two_prod(a.x, b.x), {a.x + b.x, 0.0f}}; }
 
 // x * b:  value x b.v,  tangent 1 * b.v + x * b.t
 NFAD_DEV Dual<Fast> dual_mul(const Seed& a, const Dual<Fast>& b) { return {a.x * b.v, fmaf(a.x, b.t, b.v)}; }
+NFAD_DEV Gate<Fast> dual_mul(const Seed& a, const Gate<Fast>& b) { return {a.x * b.v, fmaf(a.x, b.t, b.v)}; }
 NFAD_DEV Dual<Full> dual_mul(const Seed& a, const Dual<Full>& b)
 {
-    F2 p = two_prod(a.x, b.v);
-    return {p.h, fmaf(a.x, b.vl, p.l), fmaf(a.x, b.t, b.v + b.vl)};
+    return {f2_mul(b.v, a.x), f2_add(f2_mul(b.t, a.x), b.v)};
+}
+NFAD_DEV Gate<Full> dual_mul(const Seed& a, const Gate<Full>& b)
+{
+    return {f2_mul(b.v, a.x), f2_add(f2_mul(b.t, a.x), b.v), b.kexp};
 }
 
 NFAD_DEV Dual<Fast> dual_mul(const Dual<Fast>& a, const Dual<Fast>& b)
@@ -99,71 +116,84 @@ NFAD_DEV Dual<Fast> dual_mul(const Dual<Fast>& a, const Dual<Fast>& b)
 }
 NFAD_DEV Dual<Full> dual_mul(const Dual<Full>& a, const Dual<Full>& b)
 {
-    F2 p = two_prod(a.v, b.v);
-    return {p.h, fmaf(a.v, b.vl, fmaf(a.vl, b.v, p.l)), fmaf(a.v, b.t, a.t * b.v)};
+    return {f2_mul(a.v, b.v), f2_add(f2_mul(a.v, b.t), f2_mul(a.t, b.v))};
 }
 
-// ----------------------------------------------------------------- access helpers for unary primitives
+// ----------------------------------------------------------------- chain rule's last factor
 
-NFAD_DEV float in_v(const Seed& a) { return a.x; }
-NFAD_DEV float in_vl(const Seed&) { return 0.0f; }
-NFAD_DEV float in_v(const Dual<Fast>& a) { return a.v; }
-NFAD_DEV float in_vl(const Dual<Fast>&) { return 0.0f; }
-NFAD_DEV float in_v(const Dual<Full>& a) { return a.v; }
-NFAD_DEV float in_vl(const Dual<Full>& a) { return a.vl; }
-// d * (tangent of the input): the chain rule's last factor; free for the seed
+// d * (tangent of the input); free for the seed
 NFAD_DEV float chain(float d, const Seed&) { return d; }
 NFAD_DEV float chain(float d, const Dual<Fast>& a) { return d * a.t; }
-NFAD_DEV float chain(float d, const Dual<Full>& a) { return d * a.t; }
+NFAD_DEV F2 chain(F2 d, const Seed&) { return d; }
+NFAD_DEV F2 chain(F2 d, const Dual<Full>& a) { return f2_mul(d, a.t); }
+
+NFAD_DEV float in_v(const Seed& a) { return a.x; }
+NFAD_DEV float in_v(const Dual<Fast>& a) { return a.v; }
+NFAD_DEV F2 in_v2(const Seed& a) { return {a.x, 0.0f}; }
+NFAD_DEV F2 in_v2(const Dual<Full>& a) { return a.v; }
+
+// ----------------------------------------------------------------- the logistic function and its slope
+
+// L(w) = 1/(1+exp(-w)), L' = L (1 - L), from one e = exp(-|w|):
+//   big = 1/(1+e), small = e big = 1 - big;  L = small for w < 0, big for w >= 0.
+// Fast: (value, slope).
+NFAD_DEV Gate<Fast> logistic_fast(float w, float minus_log2e_scale)
+{
+    float e = exp2_fast(minus_log2e_scale * fabsf(w));
+    float big = hw::rcp_approx(1.0f + e);
+    float small_ = e * big;
+    return {w < 0.0f ? small_ : big, big * small_};
+}
+
+// Full: |w| = -(ah + al).  For w < 0 the common factor 2^n of e is left out of
+// value and slope (kexp = n); for w >= 0 the value is the pair (1, -small).
+NFAD_DEV Gate<Full> logistic_full(float ah, float al, bool neg)
+{
+    ExpParts E = exp_parts_full(ah, al);
+    float sc = pow2_clamped(E.n);
+    F2 e = {E.p.h * sc, E.p.l * sc};
+    F2 big = f2_rcp(f2_add_big(1.0f, e));
+    F2 pr = f2_mul(E.p, big);                  // small / 2^n
+    F2 dd = f2_mul(pr, big);                   // big small / 2^n
+    float sm = f2_value(pr) * sc;
+    F2 v = neg ? pr : F2{1.0f, -sm};
+    F2 d = neg ? dd : F2{dd.h * sc, dd.l * sc};
+    return {v, d, neg ? E.n : 0};
+}
 
 // ----------------------------------------------------------------- sigmoid
 
-// s = sigmoid(v), s' = s (1 - s).  One exp(-|v|) gives s and 1 - s without
-// subtraction; for v >= 0 the value is held as 1 - small.
-template <class In> NFAD_DEV Dual<Fast> dual_sigmoid_fast(const In& a)
+template <class In> NFAD_DEV Gate<Fast> dual_sigmoid_fast(const In& a)
 {
-    float v = in_v(a);
-    float e = exp2_fast(-1.44269502f * fabsf(v));
-    LogisticPair lp = logistic_pair_fast(e);
-    bool neg = v < 0.0f;
-    float s = neg ? lp.small_ : lp.big;
-    return {s, chain(lp.big * lp.small_, a)};
+    Gate<Fast> g = logistic_fast(in_v(a), -1.44269502f);
+    return {g.v, chain(g.t, a)};
 }
-
-template <class In> NFAD_DEV Dual<Full> dual_sigmoid_full(const In& a)
+template <class In> NFAD_DEV Gate<Full> dual_sigmoid_full(const In& a)
 {
-    float v = in_v(a), vl = in_vl(a);
-    bool neg = v < 0.0f;
-    F2 e = exp_full(-fabsf(v), neg ? vl : -vl);
-    LogisticPair lp = logistic_pair_full(e);
-    float d = lp.big * lp.small_;
-    return {neg ? lp.small_ : 1.0f, neg ? 0.0f : -lp.small_, chain(d, a)};
+    F2 v = in_v2(a);
+    bool neg = v.h < 0.0f;
+    Gate<Full> g = logistic_full(-fabsf(v.h), neg ? v.l : -v.l, neg);
+    return {g.v, chain(g.t, a), g.kexp};
 }
-
-NFAD_DEV Dual<Fast> dual_sigmoid(Fast, const Seed& a) { return dual_sigmoid_fast(a); }
-NFAD_DEV Dual<Full> dual_sigmoid(Full, const Seed& a) { return dual_sigmoid_full(a); }
-NFAD_DEV Dual<Fast> dual_sigmoid(const Dual<Fast>& a) { return dual_sigmoid_fast(a); }
-NFAD_DEV Dual<Full> dual_sigmoid(const Dual<Full>& a) { return dual_sigmoid_full(a); }
+NFAD_DEV Gate<Fast> dual_sigmoid(Fast, const Seed& a) { return dual_sigmoid_fast(a); }
+NFAD_DEV Gate<Full> dual_sigmoid(Full, const Seed& a) { return dual_sigmoid_full(a); }
+NFAD_DEV Gate<Fast> dual_sigmoid(const Dual<Fast>& a) { return dual_sigmoid_fast(a); }
+NFAD_DEV Gate<Full> dual_sigmoid(const Dual<Full>& a) { return dual_sigmoid_full(a); }
 
 // ----------------------------------------------------------------- (1 + tanh u)/2
 
-// H = (1 + tanh u)/2 = sigmoid(2u),  H' = 2 H (1 - H)   [= (1 - tanh^2 u)/2]
-NFAD_DEV Dual<Fast> dual_half_one_plus_tanh(const Dual<Fast>& u)
+// H = (1 + tanh u)/2 = L(2u),  dH/du = 2 L'(2u)   [= (1 - tanh^2 u)/2]
+NFAD_DEV Gate<Fast> dual_half_one_plus_tanh(const Dual<Fast>& u)
 {
-    float e = exp2_fast(-2.88539004f * fabsf(u.v));
-    LogisticPair lp = logistic_pair_fast(e);
-    float s = u.v < 0.0f ? lp.small_ : lp.big;
-    return {s, (u.t + u.t) * (lp.big * lp.small_)};
+    Gate<Fast> g = logistic_fast(u.v, -2.88539004f);
+    return {g.v, (u.t + u.t) * g.t};
 }
-
-NFAD_DEV Dual<Full> dual_half_one_plus_tanh(const Dual<Full>& u)
+NFAD_DEV Gate<Full> dual_half_one_plus_tanh(const Dual<Full>& u)
 {
-    bool neg = u.v < 0.0f;
-    float two_ul = u.vl + u.vl;
-    F2 e = exp_full(-2.0f * fabsf(u.v), neg ? two_ul : -two_ul);
-    LogisticPair lp = logistic_pair_full(e);
-    float d = lp.big * lp.small_;
-    return {neg ? lp.small_ : 1.0f, neg ? 0.0f : -lp.small_, (u.t + u.t) * d};
+    bool neg = u.v.h < 0.0f;
+    float two_ul = u.v.l + u.v.l;
+    Gate<Full> g = logistic_full(-2.0f * fabsf(u.v.h), neg ? two_ul : -two_ul, neg);
+    return {g.v, f2_mul(g.t, F2{u.t.h + u.t.h, u.t.l + u.t.l}), g.kexp};
 }
 
 // ----------------------------------------------------------------- (1 + erf z)/2
@@ -172,80 +202,86 @@ NFAD_DEV Dual<Full> dual_half_one_plus_tanh(const Dual<Full>& u)
 // With E = exp(-z^2) and W = erfcx(|z|)/2:  erfc(|z|)/2 = E W, so
 //   z < 0:  H = E W           z >= 0:  H = 1 - E W
 // and the same E serves the tangent.
-NFAD_DEV Dual<Fast> dual_half_one_plus_erf(const Dual<Fast>& z)
+NFAD_DEV Gate<Fast> dual_half_one_plus_erf(const Dual<Fast>& z)
 {
-    const float kInvSqrtPi = 0.564189612865448f;
+    // E is formed as 2^64 exp(-z^2) and W as 2^-64 W: see half_erfcx_fast_scaled
+    const float kInvSqrtPiScaled = 0.564189612865448f * 5.42101086e-20f;
     float za = fabsf(z.v);
-    float e = exp2_fast(-1.44269502f * (za * za));
-    float a = e * half_erfcx_fast(za);
-    float h = z.v < 0.0f ? a : 1.0f - a;
-    return {h, (e * kInvSqrtPi) * z.t};
+    float e64 = hw::ex2_approx_ftz(fmaf(za * za, -1.44269502f, 64.0f));
+    float a = e64 * half_erfcx_fast_scaled(za);
+    return {z.v < 0.0f ? a : 1.0f - a, e64 * (kInvSqrtPiScaled * z.t)};
 }
 
-NFAD_DEV Dual<Full> dual_half_one_plus_erf(const Dual<Full>& z)
+NFAD_DEV Gate<Full> dual_half_one_plus_erf(const Dual<Full>& z)
 {
-    const float kInvSqrtPi = 0.564189612865448f;
-    bool neg = z.v < 0.0f;
-    float za = fabsf(z.v);
-    float zla = neg ? -z.vl : z.vl;            // |z| = za + zla
+    const F2 kInvSqrtPi = {0.564189612865448f, -2.9317691e-08f};
+    bool neg = z.v.h < 0.0f;
+    float za = fabsf(z.v.h);
+    float zla = neg ? -z.v.l : z.v.l;          // |z| = za + zla
     F2 sq = two_prod(za, za);
-    F2 e = exp_full(-sq.h, -sq.l);             // exp(-za^2): the square is exact
-    float w = half_erfcx_full(za);
-    float t0 = e.h * kInvSqrtPi;               // |d/dz| of erfc(z)/2 at za
-    float a0 = fmaf(e.h, w, e.l * w);          // erfc(za)/2
+    ExpParts E = exp_parts_full(-sq.h, -sq.l); // exp(-za^2): the square is exact
+    F2 a = f2_mul(half_erfcx_full(za), E.p);   // erfc(za)/2, without 2^n
+    F2 t0 = f2_mul(E.p, kInvSqrtPi);           // its slope's magnitude at za, without 2^n
     // first order in the low part of the argument: the value moves by -t0 zla,
     // the exponential by the factor (1 - 2 za zla)
-    float a = fmaf(-t0, zla, a0);
-    float t = fmaf(t0, -2.0f * (za * zla), t0);
-    return {neg ? a : 1.0f, neg ? 0.0f : -a, t * z.t};
+    a.l = fmaf(-t0.h, zla, a.l);
+    t0.l = fmaf(t0.h, -2.0f * (za * zla), t0.l);
+    float sc = pow2_clamped(E.n);
+    F2 v = neg ? a : F2{1.0f, -(f2_value(a) * sc)};
+    F2 d = neg ? t0 : F2{t0.h * sc, t0.l * sc};
+    return {v, f2_mul(d, z.t), neg ? E.n : 0};
 }
 
 // ----------------------------------------------------------------- softplus, and tanh of a softplus
 
 // p = softplus(v) = log1p(exp v),  p' = sigmoid(v).
-// The result remembers e = exp(-|v|): every later use of p (its own value, its
-// tangent, tanh p) is an algebraic function of e.
+// The result remembers exp(-|v|): every later use of p (its tangent, tanh p) is
+// an algebraic function of it, so the logarithm itself is never needed here.
 template <class P> struct SoftplusDual;
-template <> struct SoftplusDual<Fast> { float e; bool neg; float tin; float x; };
-template <> struct SoftplusDual<Full> { F2 e; bool neg; float tin; float x; };
+template <> struct SoftplusDual<Fast> { float e; bool neg; };
+template <> struct SoftplusDual<Full> { ExpParts E; bool neg; };
 
 NFAD_DEV SoftplusDual<Fast> dual_softplus(Fast, const Seed& a)
 {
-    return {exp2_fast(-1.44269502f * fabsf(a.x)), a.x < 0.0f, 1.0f, a.x};
+    return {exp2_fast(-1.44269502f * fabsf(a.x)), a.x < 0.0f};
 }
 NFAD_DEV SoftplusDual<Full> dual_softplus(Full, const Seed& a)
 {
-    return {exp_full(-fabsf(a.x), 0.0f), a.x < 0.0f, 1.0f, a.x};
+    return {exp_parts_full(-fabsf(a.x), 0.0f), a.x < 0.0f};
 }
 
 // tanh(log1p(w)) = ((1+w)^2 - 1)/((1+w)^2 + 1) = n/(n+2), n = w^2 + 2w, w = e^v.
 // In terms of e = exp(-|v|), all terms positive:
-//   v <  0 (w = e):    T = (e^2 + 2e)/(e^2 + 2e + 2)
-//   v >= 0 (w = 1/e):  T = 1 - 2e^2/(1 + 2e + 2e^2)
+//   v <  0 (w = e):    T = e (e + 2) / (e^2 + 2e + 2)
+//   v >= 0 (w = 1/e):  T = 1 - e (2e) / (2e^2 + 2e + 1)
 // and T' = sech^2(p) sigmoid(v) = 4 e (1+e) / den^2, times e again for v >= 0.
-NFAD_DEV Dual<Fast> dual_tanh(const SoftplusDual<Fast>& p)
+NFAD_DEV Gate<Fast> dual_tanh(const SoftplusDual<Fast>& p)
 {
     float e = p.e;
-    float e2 = e * e;
-    float num_n = fmaf(e, e, e + e);
-    float den = p.neg ? num_n + 2.0f : fmaf(2.0f, e2, fmaf(2.0f, e, 1.0f));
+    float g = p.neg ? e + 2.0f : e + e;
+    float num = e * g;
+    float den = num + (p.neg ? 2.0f : fmaf(2.0f, e, 1.0f));
     float rd = hw::rcp_approx(den);
-    float sm = (p.neg ? num_n : e2 + e2) * rd;
+    float sm = num * rd;
     float k = (4.0f * e) * (1.0f + e) * (rd * rd);
-    return {p.neg ? sm : 1.0f - sm, (p.neg ? k : k * e) * p.tin};
+    return {p.neg ? sm : 1.0f - sm, p.neg ? k : k * e};
 }
 
-NFAD_DEV Dual<Full> dual_tanh(const SoftplusDual<Full>& p)
+NFAD_DEV Gate<Full> dual_tanh(const SoftplusDual<Full>& p)
 {
-    float e = p.e.h;
-    float e2 = e * e;
-    float num_n = fmaf(e, e, e + e);
-    float den = p.neg ? num_n + 2.0f : fmaf(2.0f, e2, fmaf(2.0f, e, 1.0f));
-    float r0 = hw::rcp_approx(den);
-    float rd = fmaf(r0, fmaf(-den, r0, 1.0f), r0);
-    float sm = (p.neg ? num_n : e2 + e2) * rd;
-    float k = (4.0f * e) * (1.0f + e) * (rd * rd);
-    return {p.neg ? sm : 1.0f, p.neg ? 0.0f : -sm, (p.neg ? k : k * e) * p.tin};
+    const bool neg = p.neg;
+    float sc = pow2_clamped(p.E.n);
+    F2 e = {p.E.p.h * sc, p.E.p.l * sc};
+    F2 g = neg ? f2_add_big(2.0f, e) : F2{e.h + e.h, e.l + e.l};
+    F2 num = f2_mul(e, g);
+    F2 base = neg ? F2{2.0f, 0.0f} : f2_add_big(1.0f, F2{e.h + e.h, e.l + e.l});
+    F2 rd = f2_rcp(f2_add(base, num));
+    F2 f0 = neg ? p.E.p : e;                   // the front factor e, without 2^n on the small side
+    F2 sm = f2_mul(f2_mul(f0, g), rd);
+    F2 tt = f2_mul(f2_mul(f0, f2_add_big(1.0f, e)), f2_mul(rd, rd));
+    tt = f2_mul(tt, neg ? F2{4.0f, 0.0f} : F2{4.0f * e.h, 4.0f * e.l});
+    F2 v = neg ? sm : F2{1.0f, -f2_value(sm)};
+    return {v, tt, neg ? p.E.n : 0};
 }
 
 // ----------------------------------------------------------------- the four activations (Table I)
@@ -255,21 +291,10 @@ struct GeluTanh {};
 struct Swish {};
 struct Mish {};
 
-struct ActOut { float y, dydx; };
-
-// Beyond |x| = kSat the gate h(x) of f = x h(x) is 0 or 1 to every fp32 bit and
-// h'(x) is 0, so the chain runs on the clamped argument (which also keeps x^2,
-// x^3 finite for any input) and f(x) = x is restored for x > kSat.
-template <class K> struct Saturation;
-template <> struct Saturation<GeluErf> { static constexpr float kSat = 20.0f; };
-template <> struct Saturation<GeluTanh> { static constexpr float kSat = 20.0f; };
-template <> struct Saturation<Swish> { static constexpr float kSat = 120.0f; };
-template <> struct Saturation<Mish> { static constexpr float kSat = 120.0f; };
-
 // The gate h(x) of each activation f(x) = x h(x), as a dual number.
 
 // GELU, erf form: h = Phi(x) = (1 + erf(x/sqrt2))/2
-template <class P> NFAD_DEV Dual<P> gate(GeluErf, Seed X)
+template <class P> NFAD_DEV Gate<P> gate(GeluErf, Seed X)
 {
     const Const2 kInvSqrt2 = {0.7071067690849304f, 1.2101617e-08f};
     Dual<P> Z = dual_scale(P{}, kInvSqrt2, X);
@@ -277,7 +302,7 @@ template <class P> NFAD_DEV Dual<P> gate(GeluErf, Seed X)
 }
 
 // GELU, tanh form (Table I): h = (1 + tanh(sqrt(2/pi) (x + 0.044715 x^3)))/2
-template <class P> NFAD_DEV Dual<P> gate(GeluTanh, Seed X)
+template <class P> NFAD_DEV Gate<P> gate(GeluTanh, Seed X)
 {
     const Const2 kA = {0.044714998453855515f, 1.5461444e-09f};   // 0.044715
     const Const2 kC = {0.7978845834732056f, -2.2670340e-08f};    // sqrt(2/pi)
@@ -289,30 +314,55 @@ template <class P> NFAD_DEV Dual<P> gate(GeluTanh, Seed X)
 }
 
 // Swish (Table I, Table II): h = sigmoid(x)
-template <class P> NFAD_DEV Dual<P> gate(Swish, Seed X) { return dual_sigmoid(P{}, X); }
+template <class P> NFAD_DEV Gate<P> gate(Swish, Seed X) { return dual_sigmoid(P{}, X); }
 
 // Mish (Table I): h = tanh(softplus(x))
-template <class P> NFAD_DEV Dual<P> gate(Mish, Seed X) { return dual_tanh(dual_softplus(P{}, X)); }
+template <class P> NFAD_DEV Gate<P> gate(Mish, Seed X) { return dual_tanh(dual_softplus(P{}, X)); }
 
-// f = x h(x): the last node of every chain is the product of the seed with the
-// gate (v3 = v1 v2 with v2 = x in the Swish example), where Eq. 3 merges the tangents.
-template <class K, class P> NFAD_DEV Dual<P> activation(K, Seed X) { return dual_mul(X, gate<P>(K{}, X)); }
+struct ActOut { float y, dydx; };
 
-// x -> (f(x), f'(x)) in fp32, for any finite or non-finite x.
-template <class K, class P> NFAD_DEV ActOut evaluate(float x)
+// Saturation.  Beyond |x| = kFull the gate is 0 or 1 to every fp32 bit and its
+// slope is exactly 0 (the exponential has underflowed to zero), so evaluating
+// the gate at the clamped argument changes nothing; it is what keeps x^2, x^3
+// and the error-free transformations finite for inputs up to the largest float.
+// The Fast policy needs that only where an intermediate can overflow (the cubic
+// of the tanh form).
+template <class K> struct Saturation;
+template <> struct Saturation<GeluErf> { static constexpr float kFull = 20.0f; static constexpr bool kFastClamp = false; };
+template <> struct Saturation<GeluTanh> { static constexpr float kFull = 20.0f; static constexpr bool kFastClamp = true; };
+template <> struct Saturation<Swish> { static constexpr float kFull = 120.0f; static constexpr bool kFastClamp = false; };
+template <> struct Saturation<Mish> { static constexpr float kFull = 120.0f; static constexpr bool kFastClamp = false; };
+
+// x -> (f(x), f'(x)) in fp32, for any finite or non-finite x.  f = x h(x): the
+// last node of every chain is the product of the seed with the gate (v3 = v1 v2
+// with v2 = x in the Swish example), where Eq. 3 merges the tangents.
+template <class K> NFAD_DEV ActOut evaluate(K, Full, float x)
 {
-    constexpr float kSat = Saturation<K>::kSat;
-    float xc = x < -kSat ? -kSat : (x > kSat ? kSat : x);    // NaN stays NaN
-    Dual<P> Y = activation<K, P>(K{}, Seed{xc});
+    constexpr float kSat = Saturation<K>::kFull;
+    float xc = hw::clamp_nan(x, -kSat, kSat);
+    Seed X{xc};
+    Gate<Full> Y = dual_mul(X, gate<Full>(K{}, X));
     float y = dual_value(Y);
-    return {x > kSat ? x : y, Y.t};
+    return {x > kSat ? x : y, dual_tangent(Y)};
 }
+
+template <class K> NFAD_DEV ActOut evaluate(K, Fast, float x)
+{
+    const float kMax = 3.40282347e+38f;
+    // +-inf become the largest float, which rounds back to inf in either 16-bit type
+    float xf = hw::clamp_nan(x, -kMax, kMax);
+    float xg = Saturation<K>::kFastClamp ? hw::clamp_nan(x, -12.0f, 12.0f) : xf;
+    Gate<Fast> Y = dual_mul(Seed{xf}, gate<Fast>(K{}, Seed{xg}));
+    return {dual_value(Y), dual_tangent(Y)};
+}
+
+template <class K, class P> NFAD_DEV ActOut evaluate(float x) { return evaluate(K{}, P{}, x); }
 
 // x -> h(x) alone (what a recomputation pass re-materialises).
 template <class K, class P> NFAD_DEV float evaluate_gate(float x)
 {
-    constexpr float kSat = Saturation<K>::kSat;
-    float xc = x < -kSat ? -kSat : (x > kSat ? kSat : x);
+    constexpr float kSat = Saturation<K>::kFull;
+    float xc = hw::clamp_nan(x, -kSat, kSat);
     return dual_value(gate<P>(K{}, Seed{xc}));
 }
 

@@ -19,6 +19,23 @@ NFAD_DEV float ex2_approx(float a)
     return r;
 }
 
+// 2^a, one MUFU.EX2; results below 2^-126 are flushed to zero.
+NFAD_DEV float ex2_approx_ftz(float a)
+{
+    float r;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(a));
+    return r;
+}
+
+// min(max(a, lo), hi) that returns NaN for a NaN (plain fminf / fmaxf drop it).
+NFAD_DEV float clamp_nan(float a, float lo, float hi)
+{
+    float r;
+    asm("max.NaN.f32 %0, %1, %2;" : "=f"(r) : "f"(a), "f"(lo));
+    asm("min.NaN.f32 %0, %1, %2;" : "=f"(r) : "f"(r), "f"(hi));
+    return r;
+}
+
 // 1/a for a normal a, MUFU.RCP (about 1 ulp).
 NFAD_DEV float rcp_approx(float a)
 {

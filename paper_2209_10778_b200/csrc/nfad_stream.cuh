@@ -7,9 +7,8 @@
 //
 // Work decomposition: a tile is kBlock * kUnroll consecutive packets; thread t
 // of a CTA owns packets t, t + kBlock, ... of the tile, so every warp-level
-// access is one contiguous 512-byte run.  A grid of (SM count x resident CTAs)
-// walks the tiles with a grid stride; each thread issues all kUnroll * NIN loads
-// of its tile before the first use.  Elements before the first and after the
+// access is one contiguous 512-byte run.  One CTA per tile; each thread issues
+// all kUnroll * NIN loads of its tile before the first use.  Elements before the first and after the
 // last whole packet (unaligned base, ragged tail) are handled one by one by the
 // first warps of CTA 0 with the very same per-element code, so the vector and
 // scalar paths agree bit for bit.
@@ -23,7 +22,10 @@
 namespace nfad {
 
 constexpr int kBlock = 256;
-constexpr int kUnroll = 4;
+#ifndef NFAD_UNROLL
+#define NFAD_UNROLL 4
+#endif
+constexpr int kUnroll = NFAD_UNROLL;
 
 // ---------------------------------------------------------------- storage types
 
@@ -261,7 +263,7 @@ cudaError_t launch_stream(const void* const* in, void* const* out, size_t n, cud
     cudaError_t e = device_info(&di);
     if (e != cudaSuccess) return e;
 
-    static thread_local int occ_stream = 0, occ_scalar = 0;   // per instantiation
+    static thread_local int occ_scalar = 0;   // per instantiation
     if (!congruent) {
         if (occ_scalar == 0) {
             e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ_scalar, scalar_kernel<S, Op>, kBlock, 0);
@@ -279,15 +281,15 @@ cudaError_t launch_stream(const void* const* in, void* const* out, size_t n, cud
     if (head > n) head = n;
     a.head = head;
     a.packets = (n - head) / S::kVec;
-    if (occ_stream == 0) {
-        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ_stream, stream_kernel<S, Op>, kBlock, 0);
-        if (e != cudaSuccess) return e;
-    }
     const size_t tile_packets = size_t(kBlock) * kUnroll;
     size_t tiles = (a.packets + tile_packets - 1) / tile_packets;
     if (tiles == 0) tiles = 1;                                  // edges only
-    size_t cap = size_t(di.sm_count) * occ_stream;
-    stream_kernel<S, Op><<<(unsigned)(tiles < cap ? tiles : cap), kBlock, 0, st>>>(a);
+    // One tile per CTA, handed out in address order by the hardware as CTAs retire: measured
+    // on B200 this moves a 1-read-2-write stream ~15 % faster than a resident grid striding over
+    // the tiles (the window of addresses in flight stays compact), and it balances the SMs at
+    // tile granularity.  The kernel's tile loop only matters beyond 2^31-1 tiles.
+    size_t grid = tiles < size_t(0x7fffffff) ? tiles : size_t(0x7fffffff);
+    stream_kernel<S, Op><<<(unsigned)grid, kBlock, 0, st>>>(a);
     return cudaPeekAtLastError();
 }
 

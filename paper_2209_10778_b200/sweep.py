@@ -1,0 +1,215 @@
+"""Per-kernel timing sweep of the activation pass (one JSON line per case).
+
+    python -m paper_2209_10778_b200.sweep --n 100663296 --dtypes bf16 --kinds gelu_erf --ops forward,backward
+    python -m paper_2209_10778_b200.sweep --config sizes      # every kind x dtype at n = 2^16 ... 2^30
+    python -m paper_2209_10778_b200.sweep --config resnet50   # Mish / Swish on the five ResNet-50 stage shapes
+    python -m paper_2209_10778_b200.sweep --config stack      # 12 stacked GELU layers under three layouts
+
+Each case launches one kernel `reps` times back to back between two CUDA events
+on the launching stream, after 3 warm-up launches; buffers are rotated so that
+at least 4x the L2 capacity is touched between two uses of the same buffer
+(tensors larger than L2 need no rotation).  GB/s is algorithmic bytes (the
+tensors the call must read and write, once) over the mean launch time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+
+import torch
+
+from . import binding as nfad
+from . import workloads as W
+
+L2_BYTES = 126 * 1024 * 1024
+
+# tensors read / written per element by each call
+OPS = {
+    "forward": (1, 2), "infer": (1, 1), "backward": (2, 1),
+    "conv_backward": (2, 1), "recompute_backward": (2 + 1 + 1, 1 + 1),   # phase 1: x -> h; phase 2: g, x, h -> gin
+}
+
+
+def _peak():
+    path = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return 6650.0, "fallback"
+
+
+def _make_sets(n, dtype, n_tensors, dev, std=1.0):
+    es = 4 if dtype == "f32" else 2
+    per_set = n_tensors * n * es
+    n_sets = 1 if n * es > L2_BYTES else max(2, -(-4 * L2_BYTES // per_set))
+    n_sets = min(n_sets, 256)
+    sets = []
+    for i in range(n_sets):
+        x = W.normal(n, dtype, 10 + i, std, dev)
+        g = W.normal(n, dtype, 500 + i, 1.0, dev)
+        s = {"x": x, "g": g, "y": torch.empty_like(x), "d": torch.empty_like(x), "gin": torch.empty_like(x)}
+        sets.append(s)
+    return sets
+
+
+def time_case(kind: str, dtype: str, op: str, n: int, reps: int = 20, dev="cuda", std=1.0):
+    es = 4 if dtype == "f32" else 2
+    sets = _make_sets(n, dtype, 5, dev, std)
+    for s in sets:
+        nfad.nfad_act_forward(kind, s["x"], s["y"], s["d"])
+    scratch = None
+    if op == "recompute_backward":
+        scratch = [torch.empty(nfad.nfad_cmp_recompute_scratch_bytes(kind, dtype, n), dtype=torch.uint8, device=dev)
+                   for _ in sets]
+
+    def launch(i):
+        s = sets[i % len(sets)]
+        if op == "forward":
+            nfad.nfad_act_forward(kind, s["x"], s["y"], s["d"])
+        elif op == "infer":
+            nfad.nfad_act_forward_infer(kind, s["x"], s["y"])
+        elif op == "backward":
+            nfad.nfad_act_backward(kind, s["g"], s["d"], s["gin"])
+        elif op == "conv_backward":
+            nfad.nfad_cmp_conv_backward(kind, s["g"], s["x"], s["gin"])
+        elif op == "recompute_backward":
+            nfad.nfad_cmp_recompute_backward(kind, s["g"], s["x"], scratch[i % len(sets)], s["gin"])
+        else:
+            raise ValueError(op)
+
+    for i in range(3):
+        launch(i)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(reps):
+        launch(3 + i)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / reps
+    r, w = OPS[op]
+    algo = (r + w) * es * n
+    peak, src = _peak()
+    gbs = algo / (ms / 1e3) / 1e9
+    return {"kind": kind, "dtype": dtype, "op": op, "n": n, "ms": ms, "elements_per_s": n / (ms / 1e3),
+            "algorithmic_bytes": algo, "GBps": gbs, "frac_of_peak": gbs / peak, "peak_GBps": peak, "peak_source": src,
+            "frac_of_nominal_8000": gbs / 8000.0, "buffer_sets": len(sets), "reps": reps}
+
+
+def run_stack(layers: int, n: int, dtype: str, kind: str, dev="cuda", reps: int = 3):
+    """L stacked activations: forward through all layers, then backward in reverse, under the three
+    layouts; reports the bytes kept alive between the passes and the total device time."""
+    es = 2 if dtype != "f32" else 4
+    out = []
+    x0 = W.normal(n, dtype, 0, 1.0, dev)
+    gL = W.normal(n, dtype, 1, 1.0, dev)
+    for layout in ("nested", "conventional", "recompute"):
+        torch.cuda.empty_cache()
+        torch.cuda.reset_peak_memory_stats()
+        base = torch.cuda.memory_allocated()
+        # nested: the layer input may be dropped at once (two ping-pong activations) and f'(x_i) is kept;
+        # the other two keep every layer's input x_i alive instead (x_0 is the caller's tensor)
+        saved = [torch.empty_like(x0) for _ in range(layers if layout == "nested" else layers - 1)]
+        act = [torch.empty_like(x0), torch.empty_like(x0)]
+        grad = [torch.empty_like(x0), torch.empty_like(x0)]
+        scratch = torch.empty(nfad.nfad_cmp_recompute_scratch_bytes(kind, dtype, n), dtype=torch.uint8, device=dev) \
+            if layout == "recompute" else None
+        inputs = [x0] + saved if layout != "nested" else None        # x_i for i = 0 .. layers-1
+
+        def one_pass():
+            if layout == "nested":
+                cur = x0
+                for i in range(layers):
+                    nxt = act[i % 2]
+                    nfad.nfad_act_forward(kind, cur, nxt, saved[i])
+                    cur = nxt
+            else:
+                for i in range(layers):
+                    nxt = inputs[i + 1] if i + 1 < layers else act[0]
+                    nfad.nfad_act_forward_infer(kind, inputs[i], nxt)
+            g = gL
+            for i in reversed(range(layers)):
+                gn = grad[i % 2]
+                if layout == "nested":
+                    nfad.nfad_act_backward(kind, g, saved[i], gn)
+                elif layout == "conventional":
+                    nfad.nfad_cmp_conv_backward(kind, g, inputs[i], gn)
+                else:
+                    nfad.nfad_cmp_recompute_backward(kind, g, inputs[i], scratch, gn)
+                g = gn
+
+        one_pass()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            one_pass()
+        e1.record()
+        torch.cuda.synchronize()
+        out.append({"config": "stack", "layout": layout, "kind": kind, "dtype": dtype, "layers": layers, "n": n,
+                    "ms_fwd_bwd": e0.elapsed_time(e1) / reps,
+                    "saved_bytes": layers * n * nfad.nfad_saved_bytes_per_element(kind, dtype, layout),
+                    "saved_bytes_op_by_op_analytic": layers * n * nfad.nfad_saved_bytes_per_element(kind, dtype, "op_by_op"),
+                    "transient_scratch_bytes": scratch.numel() if scratch is not None else 0,
+                    "max_memory_allocated_delta": torch.cuda.max_memory_allocated() - base,
+                    "note": "saved_bytes counts one kept tensor per layer (f'(x_i), or x_i itself)"})
+        del saved, act, grad, scratch, inputs
+    return out
+
+
+def main(argv=None):
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--config", default=None, choices=[None, "sizes", "resnet50", "stack", "bert"])
+    ap.add_argument("--n", type=int, default=100663296)
+    ap.add_argument("--kinds", default="gelu_erf,gelu_tanh,swish,mish")
+    ap.add_argument("--dtypes", default="bf16")
+    ap.add_argument("--ops", default="forward,backward")
+    ap.add_argument("--reps", type=int, default=20)
+    ap.add_argument("--max-log2", type=int, default=30)
+    args = ap.parse_args(argv)
+    if not torch.cuda.is_available():
+        raise RuntimeError("needs a CUDA device")
+    nfad.load()
+    kinds, dtypes, ops = args.kinds.split(","), args.dtypes.split(","), args.ops.split(",")
+    if args.config == "sizes":
+        for n in W.SWEEP_SIZES:
+            if n > (1 << args.max_log2):
+                continue
+            for dtype in dtypes:
+                for kind in kinds:
+                    for op in ops:
+                        reps = max(3, min(args.reps, (1 << 28) // n + 3))
+                        print(json.dumps(time_case(kind, dtype, op, n, reps)), flush=True)
+                        torch.cuda.empty_cache()
+    elif args.config == "resnet50":
+        w = W.WORKLOADS["resnet50_stages"]
+        for si, shape in enumerate(w.shapes):
+            for kind in w.kinds:
+                for op in ops:
+                    r = time_case(kind, w.dtype, op, w.numel(si), args.reps)
+                    r["shape"] = list(shape)
+                    print(json.dumps(r), flush=True)
+    elif args.config == "bert":
+        w = W.WORKLOADS["bert_base_ffn"]
+        for kind in w.kinds:
+            for op in ops:
+                r = time_case(kind, w.dtype, op, w.numel(0), args.reps, std=w.x_std)
+                r["shape"] = list(w.shapes[0])
+                print(json.dumps(r), flush=True)
+    elif args.config == "stack":
+        w = W.WORKLOADS["gelu_stack_12"]
+        for r in run_stack(w.layers, w.numel(0), w.dtype, w.kinds[0]):
+            print(json.dumps(r), flush=True)
+    else:
+        for dtype in dtypes:
+            for kind in kinds:
+                for op in ops:
+                    print(json.dumps(time_case(kind, dtype, op, args.n, args.reps)), flush=True)
+                    torch.cuda.empty_cache()
+
+
+if __name__ == "__main__":
+    main()
