@@ -148,6 +148,17 @@ NFAD_API size_t nfad_cmp_recompute_scratch_bytes(int kind, int dtype, size_t n);
  */
 NFAD_API int nfad_saved_bytes_per_element(int kind, int dtype, int layout);
 
+/*
+ * Traffic probe (a measurement aid with no counterpart in the paper): moves
+ * n_words 32-bit words per tensor through the same streaming kernel as the
+ * activation pass, with a read/write mix of 1:1 (o0 = a), 1:2 (o0 = a, o1 = ~a)
+ * or 2:1 (o0 = a ^ b), so that the bandwidth a given mix can reach on the device
+ * is known beside the activation kernels' numbers.  Unused tensors may be NULL.
+ * Any other mix gives NFAD_E_LAYOUT.  Same pointer, aliasing and stream rules as above.
+ */
+NFAD_API int nfad_probe_stream(int reads, int writes, const void* a, const void* b, void* o0, void* o1, size_t n_words,
+                               nfad_stream_t stream);
+
 /* The cudaError_t (as an int) behind the calling thread's last NFAD_E_CUDA; 0 if none. */
 NFAD_API int nfad_last_cuda_error(void);
 

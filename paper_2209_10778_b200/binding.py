@@ -28,6 +28,7 @@ EXPORTS = (
     "nfad_act_forward", "nfad_act_forward_infer", "nfad_act_backward",
     "nfad_cmp_conv_backward", "nfad_cmp_recompute_backward", "nfad_cmp_recompute_scratch_bytes",
     "nfad_saved_bytes_per_element", "nfad_last_cuda_error", "nfad_status_string", "nfad_version",
+    "nfad_probe_stream",
 )
 
 _lib: Optional[ctypes.CDLL] = None
@@ -61,6 +62,8 @@ def load() -> ctypes.CDLL:
         lib.nfad_cmp_recompute_scratch_bytes.argtypes = [ci, ci, sz]
         lib.nfad_cmp_recompute_scratch_bytes.restype = sz
         lib.nfad_saved_bytes_per_element.argtypes = [ci, ci, ci]
+        lib.nfad_probe_stream.argtypes = [ci, ci, vp, vp, vp, vp, sz, vp]
+        lib.nfad_probe_stream.restype = ci
         lib.nfad_last_cuda_error.argtypes = []
         lib.nfad_status_string.argtypes = [ci]
         lib.nfad_status_string.restype = ctypes.c_char_p
@@ -155,6 +158,17 @@ def nfad_saved_bytes_per_element(kind, dtype, layout) -> int:
     if rc < 0:
         raise NfadError(-rc, "nfad_saved_bytes_per_element")
     return rc
+
+
+def nfad_probe_stream(reads: int, writes: int, a: torch.Tensor, b, o0: torch.Tensor, o1) -> None:
+    """Traffic probe over fp32 tensors: 1:1 (o0 = a), 1:2 (o0 = a, o1 = ~a) or 2:1 (o0 = a ^ b)."""
+    pa = _tensor(a, "a")
+    if a.dtype != torch.float32:
+        raise TypeError("the probe takes float32 tensors")
+    with torch.cuda.device(a.device):
+        _check(load().nfad_probe_stream(int(reads), int(writes), pa, _tensor(b, "b", a) if b is not None else None,
+                                        _tensor(o0, "o0", a), _tensor(o1, "o1", a) if o1 is not None else None,
+                                        a.numel(), _stream(a)), "nfad_probe_stream")
 
 
 def nfad_version() -> str:

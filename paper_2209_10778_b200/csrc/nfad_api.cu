@@ -144,6 +144,20 @@ int nfad_cmp_recompute_backward(int kind, int dtype, const void* grad_out, const
     return run(nfad::kOpRecompute2, kind, dtype, in2, out2, n, stream);
 }
 
+int nfad_probe_stream(int reads, int writes, const void* a, const void* b, void* o0, void* o1, size_t n_words,
+                      nfad_stream_t stream)
+{
+    nfad::OpCode op;
+    if (reads == 1 && writes == 1) op = nfad::kOpProbe11;
+    else if (reads == 1 && writes == 2) op = nfad::kOpProbe12;
+    else if (reads == 2 && writes == 1) op = nfad::kOpProbe21;
+    else return NFAD_E_LAYOUT;
+    const void* in[2] = {a, b};
+    void* out[2] = {o0, o1};
+    int rc = check(0, NFAD_F32, in, reads, out, writes, n_words);
+    return rc ? rc : run(op, 0, NFAD_F32, in, out, n_words, stream);
+}
+
 int nfad_saved_bytes_per_element(int kind, int dtype, int layout)
 {
     if (kind < 0 || kind > 3) return -NFAD_E_KIND;

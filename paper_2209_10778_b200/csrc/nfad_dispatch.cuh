@@ -18,6 +18,7 @@ cudaError_t dispatch_op(OpCode op, const void* const* in, void* const* out, size
     case kOpConvBackward: return launch_stream<S, ConvBackwardOp<K, P>>(in, out, n, st);
     case kOpRecompute1:   return launch_stream<S, RecomputePhase1Op<K, P>>(in, out, n, st);
     case kOpRecompute2:   return launch_stream<S, RecomputePhase2Op<K, P>>(in, out, n, st);
+    default: break;
     }
     return cudaErrorInvalidValue;
 }

@@ -21,17 +21,16 @@
 //     dual_half_one_plus_erf(z)  = (1 + erf z)/2  = erfc(-z)/2
 //
 // Policies.  Fast (16-bit storage): a value and a tangent are one float each.
-// Full (fp32 storage): both are unevaluated sums hi + lo.  That keeps (a) the
-// bits of an exponential's argument that |arg| would amplify, (b) a result of
-// the form 1 - small as the pair (1, -small), and (c) the two addends of the
-// product rule exact enough that their cancellation for x < 0 costs nothing
-// beyond the accuracy of the exponential itself; everything is rounded once, at
+// Full (fp32 storage): values and the tangents of the polynomial part of a
+// chain are unevaluated sums hi + lo; a gate's tangent is one float.  The pairs
+// keep (a) the bits of an exponential's argument that |arg| would amplify and
+// (b) a result of the form 1 - small as (1, -small); values are rounded once, at
 // the store.
 //
 // Gates.  sigmoid, (1+tanh)/2, (1+erf)/2 and tanh(softplus) all behave like
 // exp(-|v|) on their small side.  Under Full they return a `Gate`: a dual whose
-// value and tangent share a factor 2^kexp that is applied last (it is exact),
-// so that nothing on the way is rounded in the subnormal range.
+// value and tangent share a power-of-two factor that is applied last (it is
+// exact), so that nothing on the way is rounded in the subnormal range.
 #pragma once
 
 #include "nfad_numerics.cuh"
@@ -47,7 +46,7 @@ template <> struct Dual<Full> { F2 v, t; };
 
 template <class P> struct Gate;
 template <> struct Gate<Fast> { float v, t; };
-template <> struct Gate<Full> { F2 v, t; int kexp; };     // 2^kexp (v, t)
+template <> struct Gate<Full> { F2 v; float t; float sc; int n; };   // (v, t) times sc = 2^max(n,-126), times 2^(n+126) if n < -126
 
 // A constant known to more than fp32 precision.
 struct Const2 { float h, l; };
@@ -58,16 +57,25 @@ NFAD_DEV float dual_value(const Gate<Fast>& a) { return a.v; }
 NFAD_DEV float dual_tangent(const Gate<Fast>& a) { return a.t; }
 NFAD_DEV float dual_value(const Dual<Full>& a) { return f2_value(a.v); }       // the one rounding
 NFAD_DEV float dual_tangent(const Dual<Full>& a) { return f2_value(a.t); }
-NFAD_DEV float dual_value(const Gate<Full>& a) { return scale_pow2(f2_value(a.v), a.kexp); }
-NFAD_DEV float dual_tangent(const Gate<Full>& a) { return scale_pow2(f2_value(a.t), a.kexp); }
+// The scale is a power of two: exact, unless the result is subnormal, where it is the one
+// rounding.  The second factor exists only below 2^-126 (rare, so a branch).
+NFAD_DEV float gate_rest(const Gate<Full>& a) { return pow2_clamped(a.n + 126); }
+NFAD_DEV float dual_value(const Gate<Full>& a)
+{
+    float y = f2_value(a.v) * a.sc;
+    if (a.n < -126) y *= gate_rest(a);
+    return y;
+}
+NFAD_DEV float dual_tangent(const Gate<Full>& a)
+{
+    float t = a.t * a.sc;
+    if (a.n < -126) t *= gate_rest(a);
+    return t;
+}
 
 // A gate as an ordinary dual (for further generic composition).
 NFAD_DEV Dual<Fast> as_dual(const Gate<Fast>& a) { return {a.v, a.t}; }
-NFAD_DEV Dual<Full> as_dual(const Gate<Full>& a)
-{
-    float s = pow2_clamped(a.kexp);
-    return {{a.v.h * s, a.v.l * s}, {a.t.h * s, a.t.l * s}};
-}
+NFAD_DEV Dual<Full> as_dual(const Gate<Full>& a) { return {{a.v.h * a.sc, a.v.l * a.sc}, {a.t * a.sc, 0.0f}}; }
 
 // ----------------------------------------------------------------- add, scale (linear)
 
@@ -107,7 +115,7 @@ NFAD_DEV Dual<Full> dual_mul(const Seed& a, const Dual<Full>& b)
 }
 NFAD_DEV Gate<Full> dual_mul(const Seed& a, const Gate<Full>& b)
 {
-    return {f2_mul(b.v, a.x), f2_add(f2_mul(b.t, a.x), b.v), b.kexp};
+    return {f2_mul(b.v, a.x), fmaf(a.x, b.t, b.v.h) + b.v.l, b.sc, b.n};
 }
 
 NFAD_DEV Dual<Fast> dual_mul(const Dual<Fast>& a, const Dual<Fast>& b)
@@ -124,8 +132,7 @@ NFAD_DEV Dual<Full> dual_mul(const Dual<Full>& a, const Dual<Full>& b)
 // d * (tangent of the input); free for the seed
 NFAD_DEV float chain(float d, const Seed&) { return d; }
 NFAD_DEV float chain(float d, const Dual<Fast>& a) { return d * a.t; }
-NFAD_DEV F2 chain(F2 d, const Seed&) { return d; }
-NFAD_DEV F2 chain(F2 d, const Dual<Full>& a) { return f2_mul(d, a.t); }
+NFAD_DEV float chain(float d, const Dual<Full>& a) { return fmaf(d, a.t.l, d * a.t.h); }
 
 NFAD_DEV float in_v(const Seed& a) { return a.x; }
 NFAD_DEV float in_v(const Dual<Fast>& a) { return a.v; }
@@ -137,43 +144,45 @@ NFAD_DEV F2 in_v2(const Dual<Full>& a) { return a.v; }
 // L(w) = 1/(1+exp(-w)), L' = L (1 - L), from one e = exp(-|w|):
 //   big = 1/(1+e), small = e big = 1 - big;  L = small for w < 0, big for w >= 0.
 // Fast: (value, slope).
-NFAD_DEV Gate<Fast> logistic_fast(float w, float minus_log2e_scale)
+// The slope is returned times slope_in * slope_const (the chain rule's next factor and a
+// compile-time constant, folded in here so that the 2^-64 costs no instruction).
+NFAD_DEV Gate<Fast> logistic_fast(float w, float minus_log2e_scale, float slope_in, float slope_const)
 {
-    float e = exp2_fast(minus_log2e_scale * fabsf(w));
-    float big = hw::rcp_approx(1.0f + e);
-    float small_ = e * big;
-    return {w < 0.0f ? small_ : big, big * small_};
+    float e64 = exp2_fast_times_2p64(fmaf(fabsf(w), minus_log2e_scale, 64.0f));   // 2^64 e
+    float big = hw::rcp_approx(fmaf(e64, kTwoPowMinus64, 1.0f));
+    float small64 = e64 * big;                                                    // 2^64 small
+    return {w < 0.0f ? small64 * kTwoPowMinus64 : big, (small64 * big) * (slope_in * (slope_const * kTwoPowMinus64))};
 }
 
 // Full: |w| = -(ah + al).  For w < 0 the common factor 2^n of e is left out of
-// value and slope (kexp = n); for w >= 0 the value is the pair (1, -small).
+// value and slope (they carry it as `sc`); for w >= 0 the value is the pair (1, -small).
 NFAD_DEV Gate<Full> logistic_full(float ah, float al, bool neg)
 {
     ExpParts E = exp_parts_full(ah, al);
     float sc = pow2_clamped(E.n);
-    F2 e = {E.p.h * sc, E.p.l * sc};
-    F2 big = f2_rcp(f2_add_big(1.0f, e));
+    float eh = E.p.h * sc;
+    float dh = 1.0f + eh;
+    float dl = fmaf(E.p.l, sc, eh - (dh - 1.0f));   // 1 + e = dh + dl
+    F2 big = f2_rcp(F2{dh, dl});               // 1/(1+e)
     F2 pr = f2_mul(E.p, big);                  // small / 2^n
-    F2 dd = f2_mul(pr, big);                   // big small / 2^n
-    float sm = f2_value(pr) * sc;
-    F2 v = neg ? pr : F2{1.0f, -sm};
-    F2 d = neg ? dd : F2{dd.h * sc, dd.l * sc};
-    return {v, d, neg ? E.n : 0};
+    float dd = fmaf(pr.h, big.h, fmaf(pr.l, big.h, pr.h * big.l));   // big small / 2^n, one rounding
+    F2 v = neg ? pr : F2{1.0f, -(f2_value(pr) * sc)};
+    float d = neg ? dd : dd * sc;
+    return {v, d, neg ? sc : 1.0f, neg ? E.n : 0};
 }
 
 // ----------------------------------------------------------------- sigmoid
 
 template <class In> NFAD_DEV Gate<Fast> dual_sigmoid_fast(const In& a)
 {
-    Gate<Fast> g = logistic_fast(in_v(a), -1.44269502f);
-    return {g.v, chain(g.t, a)};
+    return logistic_fast(in_v(a), -1.44269502f, chain(1.0f, a), 1.0f);
 }
 template <class In> NFAD_DEV Gate<Full> dual_sigmoid_full(const In& a)
 {
     F2 v = in_v2(a);
     bool neg = v.h < 0.0f;
     Gate<Full> g = logistic_full(-fabsf(v.h), neg ? v.l : -v.l, neg);
-    return {g.v, chain(g.t, a), g.kexp};
+    return {g.v, chain(g.t, a), g.sc, g.n};
 }
 NFAD_DEV Gate<Fast> dual_sigmoid(Fast, const Seed& a) { return dual_sigmoid_fast(a); }
 NFAD_DEV Gate<Full> dual_sigmoid(Full, const Seed& a) { return dual_sigmoid_full(a); }
@@ -185,15 +194,14 @@ NFAD_DEV Gate<Full> dual_sigmoid(const Dual<Full>& a) { return dual_sigmoid_full
 // H = (1 + tanh u)/2 = L(2u),  dH/du = 2 L'(2u)   [= (1 - tanh^2 u)/2]
 NFAD_DEV Gate<Fast> dual_half_one_plus_tanh(const Dual<Fast>& u)
 {
-    Gate<Fast> g = logistic_fast(u.v, -2.88539004f);
-    return {g.v, (u.t + u.t) * g.t};
+    return logistic_fast(u.v, -2.88539004f, u.t, 2.0f);
 }
 NFAD_DEV Gate<Full> dual_half_one_plus_tanh(const Dual<Full>& u)
 {
     bool neg = u.v.h < 0.0f;
     float two_ul = u.v.l + u.v.l;
     Gate<Full> g = logistic_full(-2.0f * fabsf(u.v.h), neg ? two_ul : -two_ul, neg);
-    return {g.v, f2_mul(g.t, F2{u.t.h + u.t.h, u.t.l + u.t.l}), g.kexp};
+    return {g.v, chain(g.t + g.t, u), g.sc, g.n};
 }
 
 // ----------------------------------------------------------------- (1 + erf z)/2
@@ -207,7 +215,7 @@ NFAD_DEV Gate<Fast> dual_half_one_plus_erf(const Dual<Fast>& z)
     // E is formed as 2^64 exp(-z^2) and W as 2^-64 W: see half_erfcx_fast_scaled
     const float kInvSqrtPiScaled = 0.564189612865448f * 5.42101086e-20f;
     float za = fabsf(z.v);
-    float e64 = hw::ex2_approx_ftz(fmaf(za * za, -1.44269502f, 64.0f));
+    float e64 = exp2_fast_times_2p64(fmaf(za * za, -1.44269502f, 64.0f));
     float a = e64 * half_erfcx_fast_scaled(za);
     return {z.v < 0.0f ? a : 1.0f - a, e64 * (kInvSqrtPiScaled * z.t)};
 }
@@ -221,15 +229,15 @@ NFAD_DEV Gate<Full> dual_half_one_plus_erf(const Dual<Full>& z)
     F2 sq = two_prod(za, za);
     ExpParts E = exp_parts_full(-sq.h, -sq.l); // exp(-za^2): the square is exact
     F2 a = f2_mul(half_erfcx_full(za), E.p);   // erfc(za)/2, without 2^n
-    F2 t0 = f2_mul(E.p, kInvSqrtPi);           // its slope's magnitude at za, without 2^n
+    float t0 = f2_value(f2_mul(E.p, kInvSqrtPi));   // its slope's magnitude at za, without 2^n
     // first order in the low part of the argument: the value moves by -t0 zla,
     // the exponential by the factor (1 - 2 za zla)
-    a.l = fmaf(-t0.h, zla, a.l);
-    t0.l = fmaf(t0.h, -2.0f * (za * zla), t0.l);
+    a.l = fmaf(-t0, zla, a.l);
+    t0 = fmaf(t0, -2.0f * (za * zla), t0);
     float sc = pow2_clamped(E.n);
     F2 v = neg ? a : F2{1.0f, -(f2_value(a) * sc)};
-    F2 d = neg ? t0 : F2{t0.h * sc, t0.l * sc};
-    return {v, f2_mul(d, z.t), neg ? E.n : 0};
+    float d = neg ? t0 : t0 * sc;
+    return {v, chain(d, z), neg ? sc : 1.0f, neg ? E.n : 0};
 }
 
 // ----------------------------------------------------------------- softplus, and tanh of a softplus
@@ -243,7 +251,7 @@ template <> struct SoftplusDual<Full> { ExpParts E; bool neg; };
 
 NFAD_DEV SoftplusDual<Fast> dual_softplus(Fast, const Seed& a)
 {
-    return {exp2_fast(-1.44269502f * fabsf(a.x)), a.x < 0.0f};
+    return {exp2_fast_times_2p64(fmaf(fabsf(a.x), -1.44269502f, 64.0f)) * kTwoPowMinus64, a.x < 0.0f};
 }
 NFAD_DEV SoftplusDual<Full> dual_softplus(Full, const Seed& a)
 {
@@ -272,16 +280,21 @@ NFAD_DEV Gate<Full> dual_tanh(const SoftplusDual<Full>& p)
     const bool neg = p.neg;
     float sc = pow2_clamped(p.E.n);
     F2 e = {p.E.p.h * sc, p.E.p.l * sc};
-    F2 g = neg ? f2_add_big(2.0f, e) : F2{e.h + e.h, e.l + e.l};
+    F2 e2 = {e.h + e.h, e.l + e.l};
+    F2 g = neg ? f2_add_big(2.0f, e) : e2;
     F2 num = f2_mul(e, g);
-    F2 base = neg ? F2{2.0f, 0.0f} : f2_add_big(1.0f, F2{e.h + e.h, e.l + e.l});
-    F2 rd = f2_rcp(f2_add(base, num));
+    F2 base = neg ? F2{2.0f, 0.0f} : f2_add_big(1.0f, e2);
+    F2 den = f2_add(base, num);
+    F2 rd = f2_rcp(den);                       // 1/den
     F2 f0 = neg ? p.E.p : e;                   // the front factor e, without 2^n on the small side
     F2 sm = f2_mul(f2_mul(f0, g), rd);
-    F2 tt = f2_mul(f2_mul(f0, f2_add_big(1.0f, e)), f2_mul(rd, rd));
-    tt = f2_mul(tt, neg ? F2{4.0f, 0.0f} : F2{4.0f * e.h, 4.0f * e.l});
+    F2 ope = f2_add_big(1.0f, e);
+    F2 a1 = f2_mul(f0, ope);                                // e (1 + e)
+    F2 rd2 = two_prod(rd.h, rd.h);
+    rd2.l = fmaf(rd.h + rd.h, rd.l, rd2.l);                 // 1/den^2
+    float tt = f2_value(f2_mul(a1, rd2)) * (neg ? 4.0f : 4.0f * e.h);
     F2 v = neg ? sm : F2{1.0f, -f2_value(sm)};
-    return {v, tt, neg ? p.E.n : 0};
+    return {v, tt, neg ? sc : 1.0f, neg ? p.E.n : 0};
 }
 
 // ----------------------------------------------------------------- the four activations (Table I)
@@ -349,10 +362,17 @@ template <class K> NFAD_DEV ActOut evaluate(K, Full, float x)
 template <class K> NFAD_DEV ActOut evaluate(K, Fast, float x)
 {
     const float kMax = 3.40282347e+38f;
+    if (Saturation<K>::kFastClamp) {
+        // the gate and the tangent's product see the clamped argument (the slope is exactly 0
+        // beyond it); the value's product sees x itself, kept finite on the side where the
+        // gate is 0 so that -inf gives -0
+        float xg = hw::clamp_nan(x, -12.0f, 12.0f);
+        Gate<Fast> H = gate<Fast>(K{}, Seed{xg});
+        return {hw::max_nan(x, -kMax) * H.v, fmaf(xg, H.t, H.v)};
+    }
     // +-inf become the largest float, which rounds back to inf in either 16-bit type
     float xf = hw::clamp_nan(x, -kMax, kMax);
-    float xg = Saturation<K>::kFastClamp ? hw::clamp_nan(x, -12.0f, 12.0f) : xf;
-    Gate<Fast> Y = dual_mul(Seed{xf}, gate<Fast>(K{}, Seed{xg}));
+    Gate<Fast> Y = dual_mul(Seed{xf}, gate<Fast>(K{}, Seed{xf}));
     return {dual_value(Y), dual_tangent(Y)};
 }
 

@@ -36,6 +36,14 @@ NFAD_DEV float clamp_nan(float a, float lo, float hi)
     return r;
 }
 
+// max(a, lo) that returns NaN for a NaN.
+NFAD_DEV float max_nan(float a, float lo)
+{
+    float r;
+    asm("max.NaN.f32 %0, %1, %2;" : "=f"(r) : "f"(a), "f"(lo));
+    return r;
+}
+
 // 1/a for a normal a, MUFU.RCP (about 1 ulp).
 NFAD_DEV float rcp_approx(float a)
 {

@@ -114,7 +114,7 @@ NFAD_DEV float scale_pow2(float v, int n)
 
 // ---------------------------------------------------------------- exp, Full
 
-// e^(ah+al) = 2^n (p.h + p.l), p in [0.70, 1.42], for ah <= 0 (|al| tiny
+// e^(ah+al) = 2^n (p.h + p.l), p in [0.70, 1.42], for -300 < ah <= 0 (|al| tiny
 // against ah).  The power of two is NOT applied: callers multiply by it last,
 // where it is exact, so that a result near or below 2^-126 is rounded once.
 // Cody-Waite reduction a = n ln2 + r with the reduced argument kept as a pair, a
@@ -128,7 +128,6 @@ NFAD_DEV ExpParts exp_parts_full(float ah, float al)
     const float kMagic = 12582912.0f;          // 1.5 * 2^23: adding it rounds to an integer
     const float kLn2Hi = 0.693147182f;         // 0x3f317218
     const float kLn2Lo = -1.90465421e-09f;     // ln2 - kLn2Hi
-    ah = ah < -170.0f ? -170.0f : ah;
     float t = fmaf(ah, kLog2e, kMagic);
     float n = t - kMagic;
     int ni = hw::float_as_int(t) - 0x4B400000;
@@ -142,7 +141,7 @@ NFAD_DEV ExpParts exp_parts_full(float ah, float al)
     q = fmaf(q, r, 0.0416665077f);
     q = fmaf(q, r, 0.166666672f);
     q = fmaf(q, r, 0.5f);
-    float w = fmaf(r * r, q, dl);              // e^(r+dl) - 1 - r, to first order in dl
+    float w = fmaf(r * r, q, dl);              // e^(r+dl) - 1 - r, to first order in dl (|dl| < 2^-25)
     F2 g = fast_two_sum(r, w);
     float ph = 1.0f + g.h;
     float pl = (g.h - (ph - 1.0f)) + g.l;      // 1 + g = ph + pl exactly (|g.h| < 1)
@@ -151,8 +150,6 @@ NFAD_DEV ExpParts exp_parts_full(float ah, float al)
 
 // ---------------------------------------------------------------- exp, Fast
 
-// 2^a, a <= 0 (the caller has folded log2 e into a); keeps subnormal results.
-NFAD_DEV float exp2_fast(float a) { return hw::ex2_approx(a); }
 
 // ---------------------------------------------------------------- scaled complementary error function
 
@@ -183,26 +180,32 @@ NFAD_DEV F2 half_erfcx_full(float z)
     return f2_mul(s, r);
 }
 
-// Fast policy: the same fit at degree 8, with every coefficient pre-multiplied
-// by 2^-64.  The caller's exponential carries the matching 2^+64 (so that it
-// cannot underflow in MUFU's flush-to-zero range) and the product of the two is
-// the first place where a result may become subnormal.  Returns 2^-64 W(z).
+// Fast policy: a degree-6 fit of the same function, weighted so that both W and the
+// combination W - z/sqrt(pi) (which carries the cancellation of the GELU derivative for
+// x < 0) keep a relative error below 2^-16, with every coefficient pre-multiplied by 2^-64.
+// The caller's exponential carries the matching 2^+64 (so that it cannot underflow in
+// MUFU's flush-to-zero range) and the product of the two is the first place where a result
+// may become subnormal.  Returns 2^-64 W(z).
 NFAD_DEV float half_erfcx_fast_scaled(float z)
 {
     const float k = 2.1213202476501465f;
     const float s = 5.42101086e-20f;           // 2^-64
     float r = hw::rcp_approx(z + k);
     float q = fmaf(-2.0f * k, r, 1.0f);
-    float p = -0.00018698952f * s;
-    p = fmaf(p, q, -0.000633997901f * s);
-    p = fmaf(p, q, 0.000762930082f * s);
-    p = fmaf(p, q, 0.00489306729f * s);
-    p = fmaf(p, q, -0.00741203828f * s);
-    p = fmaf(p, q, -0.0334145501f * s);
-    p = fmaf(p, q, 0.162648439f * s);
-    p = fmaf(p, q, -0.360152334f * s);
-    p = fmaf(p, q, 0.515540004f * s);
+    float p = 0.000961262616f * s;
+    p = fmaf(p, q, 0.00436418364f * s);
+    p = fmaf(p, q, -0.00761994533f * s);
+    p = fmaf(p, q, -0.0332778953f * s);
+    p = fmaf(p, q, 0.162689358f * s);
+    p = fmaf(p, q, -0.36016348f * s);
+    p = fmaf(p, q, 0.515539289f * s);
     return p * r;
 }
+
+// Fast exponential of a non-positive argument given in base 2: one MUFU.EX2 on the
+// argument raised by 64, so that the flush-to-zero unit never sees a result below 2^-126
+// until the true value is below 2^-190.  Returns 2^64 2^a.
+constexpr float kTwoPowMinus64 = 5.42101086e-20f;
+NFAD_DEV float exp2_fast_times_2p64(float a_plus_64) { return hw::ex2_approx_ftz(a_plus_64); }
 
 }  // namespace nfad

@@ -10,6 +10,7 @@ namespace nfad {
 // Forward, training: x -> (y = f(x), f'(x)).  One pass over dual numbers; f'(x)
 // is the only tensor kept for back-propagation (Section II-C, approach 3).
 template <class K, class P> struct ForwardTrainOp {
+    static constexpr bool kPacketFixup = false;
     static constexpr int kIn = 1, kOut = 2;
     static __device__ __forceinline__ constexpr bool keep(int k) { return k == 0; }   // y is consumed next; f' much later
     static __device__ __forceinline__ void apply(const float (&in)[1], float (&out)[2])
@@ -22,6 +23,7 @@ template <class K, class P> struct ForwardTrainOp {
 
 // Forward, inference: x -> y.  Same chain; the tangent parts are dead code.
 template <class K, class P> struct ForwardInferOp {
+    static constexpr bool kPacketFixup = false;
     static constexpr int kIn = 1, kOut = 1;
     static __device__ __forceinline__ constexpr bool keep(int) { return true; }
     static __device__ __forceinline__ void apply(const float (&in)[1], float (&out)[1])
@@ -35,27 +37,45 @@ template <class K, class P> struct ForwardInferOp {
 // shares fp32's exponent range, so only there can a product land below 2^-126,
 // where it is re-formed in fp64 and rounded straight to the bf16 subnormal grid
 // (multiples of 2^-133) to keep the result a single rounding of the true product.
+// That case is rare, so it is tested once per packet and handled out of line.
+static __device__ __noinline__ float bf16_tiny_product(float g, float d)
+{
+    const double kGrid = 6.2038417431289079e-25;   // 1.5 * 2^-81: its ulp is 2^-133
+    double pd = (double)g * (double)d;
+    pd = (pd + kGrid) - kGrid;
+    return (float)pd;
+}
+
 template <bool kBf16> struct BackwardOp {
     static constexpr int kIn = 2, kOut = 1;
+    static constexpr bool kPacketFixup = kBf16;
     static __device__ __forceinline__ constexpr bool keep(int) { return true; }
-    static __device__ __forceinline__ void apply(const float (&in)[2], float (&out)[1])
+    static __device__ __forceinline__ void apply(const float (&in)[2], float (&out)[1]) { out[0] = in[0] * in[1]; }
+    // scalar path (edges): the same result, element by element
+    static __device__ __forceinline__ void apply_checked(const float (&in)[2], float (&out)[1])
     {
         float p = in[0] * in[1];
-        if (kBf16) {
-            if (fabsf(p) <= 1.17549435e-38f) {
-                const double kGrid = 6.2038417431289079e-25;   // 1.5 * 2^-81: ulp is 2^-133
-                double pd = (double)in[0] * (double)in[1];
-                pd = (pd + kGrid) - kGrid;
-                p = (float)pd;
-            }
-        }
+        if (kBf16 && fabsf(p) <= 1.17549435e-38f) p = bf16_tiny_product(in[0], in[1]);
         out[0] = p;
+    }
+    template <int V>
+    static __device__ __forceinline__ void fixup(const float (&vin)[2][V], float (&vout)[1][V])
+    {
+        bool tiny = false;
+#pragma unroll
+        for (int e = 0; e < V; ++e) tiny |= fabsf(vout[0][e]) <= 1.17549435e-38f;
+        if (tiny) {
+#pragma unroll                          // (a rolled loop would index the register arrays dynamically)
+            for (int e = 0; e < V; ++e)
+                if (fabsf(vout[0][e]) <= 1.17549435e-38f) vout[0][e] = bf16_tiny_product(vin[0][e], vin[1][e]);
+        }
     }
 };
 
 // Conventional layout: x is saved, and backward re-derives f'(x) with the full
 // transcendental chain before the multiply.
 template <class K, class P> struct ConvBackwardOp {
+    static constexpr bool kPacketFixup = false;
     static constexpr int kIn = 2, kOut = 1;
     static __device__ __forceinline__ constexpr bool keep(int) { return true; }
     static __device__ __forceinline__ void apply(const float (&in)[2], float (&out)[1])
@@ -69,6 +89,7 @@ template <class K, class P> struct ConvBackwardOp {
 // per-operator backward rules need (the gate h = v1 of the Swish example), then
 // walks those rules: x' = g v1 + g v2 v1' with v2 = x (Eq. 2).
 template <class K, class P> struct RecomputePhase1Op {
+    static constexpr bool kPacketFixup = false;
     static constexpr int kIn = 1, kOut = 1;
     static __device__ __forceinline__ constexpr bool keep(int) { return true; }
     static __device__ __forceinline__ void apply(const float (&in)[1], float (&out)[1])
@@ -109,6 +130,7 @@ template <> struct GateSlope<Mish> {
 };
 
 template <class K, class P> struct RecomputePhase2Op {
+    static constexpr bool kPacketFixup = false;
     static constexpr int kIn = 3, kOut = 1;            // grad_out, x, h
     static __device__ __forceinline__ constexpr bool keep(int) { return true; }
     static __device__ __forceinline__ void apply(const float (&in)[3], float (&out)[1])
@@ -116,6 +138,21 @@ template <class K, class P> struct RecomputePhase2Op {
         float g = in[0], x = in[1], h = in[2];
         float hs = GateSlope<K>::of(x, h);
         out[0] = fmaf(g * x, hs, g * h);
+    }
+};
+
+// Traffic probe: moves bytes through the same streaming engine with no arithmetic to speak
+// of, to measure what a given read/write mix can reach on the device.
+template <int NIN, int NOUT> struct ProbeOp {
+    static constexpr bool kPacketFixup = false;
+    static constexpr int kIn = NIN, kOut = NOUT;
+    static __device__ __forceinline__ constexpr bool keep(int k) { return k == 0; }
+    static __device__ __forceinline__ void apply(const float (&in)[NIN], float (&out)[NOUT])
+    {
+        float v = in[0];
+        if (NIN > 1) v = __uint_as_float(__float_as_uint(v) ^ __float_as_uint(in[1]));
+        out[0] = v;
+        if (NOUT > 1) out[1] = __uint_as_float(~__float_as_uint(v));
     }
 };
 

@@ -26,12 +26,23 @@ constexpr int kBlock = 256;
 #define NFAD_UNROLL 4
 #endif
 constexpr int kUnroll = NFAD_UNROLL;
+// Resident CTAs per SM the compiler must leave room for (a register cap).  The 16-bit kernels
+// are issue-bound with short dependency chains through MUFU: 5 CTAs (40 warps, <= 48 registers)
+// measured 3-5 % faster than the 4 the compiler picks by itself (7 or more spill and lose 30 %); the fp32 kernels need their
+// ~48 registers (a tighter cap spills).
+#ifndef NFAD_MIN_BLOCKS_16
+#define NFAD_MIN_BLOCKS_16 5
+#endif
+#ifndef NFAD_MIN_BLOCKS_32
+#define NFAD_MIN_BLOCKS_32 5
+#endif
 
 // ---------------------------------------------------------------- storage types
 
 struct StoreF32 {
     using elem = float;
     static constexpr int kVec = 4;             // elements per 16-byte packet
+    static constexpr int kMinBlocks = NFAD_MIN_BLOCKS_32;
     static __device__ __forceinline__ void unpack(const uint4& p, float (&v)[4])
     {
         v[0] = __uint_as_float(p.x); v[1] = __uint_as_float(p.y);
@@ -48,6 +59,7 @@ struct StoreF32 {
 struct StoreBF16 {
     using elem = __nv_bfloat16;
     static constexpr int kVec = 8;
+    static constexpr int kMinBlocks = NFAD_MIN_BLOCKS_16;
     // a bf16 is the upper half of an fp32: widening is a shift or a mask
     static __device__ __forceinline__ void unpack(const uint4& p, float (&v)[8])
     {
@@ -74,6 +86,7 @@ struct StoreBF16 {
 struct StoreF16 {
     using elem = __half;
     static constexpr int kVec = 8;
+    static constexpr int kMinBlocks = NFAD_MIN_BLOCKS_16;
     static __device__ __forceinline__ void unpack(const uint4& p, float (&v)[8])
     {
         const uint32_t w[4] = {p.x, p.y, p.z, p.w};
@@ -121,8 +134,11 @@ template <int NIN, int NOUT> struct StreamArgs {
 };
 
 // Op: struct with
-//   static constexpr int kIn, kOut;  static constexpr bool kKeep[kOut];
+//   static constexpr int kIn, kOut;  static constexpr bool keep(int out_slot);
 //   static __device__ void apply(const float (&in)[kIn], float (&out)[kOut]);
+//   static constexpr bool kPacketFixup; if set, fixup(vin, vout) may patch a whole packet's
+//   results after apply (a rare case kept off the per-element path) and apply_checked is the
+//   one-element form that includes the patch.
 template <class S, class Op>
 __device__ __forceinline__ void scalar_element(const StreamArgs<Op::kIn, Op::kOut>& a, size_t i)
 {
@@ -130,7 +146,8 @@ __device__ __forceinline__ void scalar_element(const StreamArgs<Op::kIn, Op::kOu
     float in[Op::kIn], out[Op::kOut];
 #pragma unroll
     for (int k = 0; k < Op::kIn; ++k) in[k] = S::load1(static_cast<const E*>(a.in[k]) + i);
-    Op::apply(in, out);
+    if constexpr (Op::kPacketFixup) Op::apply_checked(in, out);
+    else Op::apply(in, out);
 #pragma unroll
     for (int k = 0; k < Op::kOut; ++k) S::store1(static_cast<E*>(a.out[k]) + i, out[k]);
 }
@@ -153,6 +170,7 @@ __device__ __forceinline__ void packet_compute_store(const StreamArgs<Op::kIn, O
 #pragma unroll
         for (int k = 0; k < Op::kOut; ++k) vout[k][e] = out[k];
     }
+    if constexpr (Op::kPacketFixup) Op::template fixup<V>(vin, vout);
     const size_t byte_off = a.head * sizeof(typename S::elem);
 #pragma unroll
     for (int k = 0; k < Op::kOut; ++k) {
@@ -164,7 +182,7 @@ __device__ __forceinline__ void packet_compute_store(const StreamArgs<Op::kIn, O
 }
 
 template <class S, class Op>
-__global__ void __launch_bounds__(kBlock) stream_kernel(const StreamArgs<Op::kIn, Op::kOut> a)
+__global__ void __launch_bounds__(kBlock, S::kMinBlocks) stream_kernel(const StreamArgs<Op::kIn, Op::kOut> a)
 {
     constexpr int V = S::kVec;
     const size_t byte_off = a.head * sizeof(typename S::elem);

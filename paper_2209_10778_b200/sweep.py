@@ -4,6 +4,7 @@
     python -m paper_2209_10778_b200.sweep --config sizes      # every kind x dtype at n = 2^16 ... 2^30
     python -m paper_2209_10778_b200.sweep --config resnet50   # Mish / Swish on the five ResNet-50 stage shapes
     python -m paper_2209_10778_b200.sweep --config stack      # 12 stacked GELU layers under three layouts
+    python -m paper_2209_10778_b200.sweep --config probe      # plain 1:1 / 1:2 / 2:1 traffic through the same engine
 
 Each case launches one kernel `reps` times back to back between two CUDA events
 on the launching stream, after 3 warm-up launches; buffers are rotated so that
@@ -99,6 +100,36 @@ def time_case(kind: str, dtype: str, op: str, n: int, reps: int = 20, dev="cuda"
             "frac_of_nominal_8000": gbs / 8000.0, "buffer_sets": len(sets), "reps": reps}
 
 
+def run_probe(n_words: int, reps: int = 20, dev="cuda"):
+    """Bandwidth of plain 1:1, 1:2 and 2:1 read/write mixes through the streaming engine, and of
+    cudaMemcpy-like torch copy_, on tensors of n_words fp32 words each."""
+    out = []
+    a = torch.randn(n_words, device=dev)
+    b = torch.randn(n_words, device=dev)
+    o0 = torch.empty_like(a)
+    o1 = torch.empty_like(a)
+    peak, src = _peak()
+    cases = [("probe 1R:1W", 2, lambda: nfad.nfad_probe_stream(1, 1, a, None, o0, None)),
+             ("probe 1R:2W (forward's mix)", 3, lambda: nfad.nfad_probe_stream(1, 2, a, None, o0, o1)),
+             ("probe 2R:1W (backward's mix)", 3, lambda: nfad.nfad_probe_stream(2, 1, a, b, o0, None)),
+             ("torch copy_ 1R:1W", 2, lambda: o0.copy_(a))]
+    for name, tensors, fn in cases:
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / reps
+        gbs = tensors * 4 * n_words / (ms / 1e3) / 1e9
+        out.append({"config": "probe", "case": name, "bytes_per_tensor": 4 * n_words, "ms": ms, "GBps": gbs,
+                    "frac_of_peak": gbs / peak, "peak_GBps": peak, "peak_source": src})
+    return out
+
+
 def run_stack(layers: int, n: int, dtype: str, kind: str, dev="cuda", reps: int = 3):
     """L stacked activations: forward through all layers, then backward in reverse, under the three
     layouts; reports the bytes kept alive between the passes and the total device time."""
@@ -162,7 +193,7 @@ def run_stack(layers: int, n: int, dtype: str, kind: str, dev="cuda", reps: int 
 
 def main(argv=None):
     ap = argparse.ArgumentParser()
-    ap.add_argument("--config", default=None, choices=[None, "sizes", "resnet50", "stack", "bert"])
+    ap.add_argument("--config", default=None, choices=[None, "sizes", "resnet50", "stack", "bert", "probe"])
     ap.add_argument("--n", type=int, default=100663296)
     ap.add_argument("--kinds", default="gelu_erf,gelu_tanh,swish,mish")
     ap.add_argument("--dtypes", default="bf16")
@@ -199,6 +230,9 @@ def main(argv=None):
                 r = time_case(kind, w.dtype, op, w.numel(0), args.reps, std=w.x_std)
                 r["shape"] = list(w.shapes[0])
                 print(json.dumps(r), flush=True)
+    elif args.config == "probe":
+        for r in run_probe(args.n // 2, args.reps):          # n bf16-sized elements -> n/2 words
+            print(json.dumps(r), flush=True)
     elif args.config == "stack":
         w = W.WORKLOADS["gelu_stack_12"]
         for r in run_stack(w.layers, w.numel(0), w.dtype, w.kinds[0]):

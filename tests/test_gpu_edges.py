@@ -157,7 +157,7 @@ def test_recompute_comparator(kind, dtype):
     gw, xw = oracle.widen(dtype, W.raw_numpy(g)), oracle.widen(dtype, W.raw_numpy(x))
     got = oracle.widen(dtype, W.raw_numpy(gin))
     eps = {"f32": 2.0 ** -23, "bf16": 2.0 ** -8, "f16": 2.0 ** -11}[dtype]
-    tol = np.abs(gw) * eps * 4 * (1 + 2 * np.abs(xw)) + eps * np.abs(gw * fp)
+    tol = np.abs(gw) * eps * (4 + 8 * np.abs(xw) * (1 + xw * xw / 4)) + eps * np.abs(gw * fp)
     assert (np.abs(got - gw * fp) <= tol).all()
     with pytest.raises(nfad.NfadError) as e:
         nfad.nfad_cmp_recompute_backward(kind, g, x, scratch[:16], gin)
