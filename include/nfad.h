@@ -70,7 +70,8 @@ typedef enum {
     NFAD_E_CUDA = 5,     /* a CUDA call failed: see nfad_last_cuda_error()            */
     NFAD_E_ALIGN = 6,    /* a pointer is not a multiple of the element size           */
     NFAD_E_SCRATCH = 7,  /* scratch_bytes is smaller than the comparator needs        */
-    NFAD_E_LAYOUT = 8    /* layout is not an nfad_layout                              */
+    NFAD_E_LAYOUT = 8,   /* layout is not an nfad_layout                              */
+    NFAD_E_TOO_LARGE = 9 /* the tensors need more than the library's built-in scratch */
 } nfad_status;
 
 /* How the tensor needed by backward is kept between the passes (Section II-C). */
@@ -134,6 +135,39 @@ NFAD_API int nfad_cmp_conv_backward(int kind, int dtype, const void* grad_out, c
  */
 NFAD_API int nfad_cmp_recompute_backward(int kind, int dtype, const void* grad_out, const void* x, void* scratch,
                                 size_t scratch_bytes, void* grad_in, size_t n, nfad_stream_t stream);
+
+/*
+ * The recomputation comparator for callers that cannot hand over scratch memory.
+ * (The paper has no counterpart: this is a convenience of this library.)
+ *
+ * Some users of this code have no way to allocate device memory at the point
+ * where they call it: a plug-in running under a host application that hands out
+ * all device memory up front and forbids cudaMalloc afterwards, a serving loop in
+ * which an allocation's implicit device-wide synchronisation would stall every
+ * other stream, or a component that is simply not given an allocator.  For them
+ * this entry point does what nfad_cmp_recompute_backward does, bit for bit, but
+ * takes its scratch from a fixed array of NFAD_NOALLOC_SCRATCH_BYTES that is part
+ * of the library image (every GPU that loads the library holds those bytes
+ * until the process exits).  It calls no allocation routine of any kind.
+ *
+ *   grad_out, x [in], grad_in [out]: n elements each, same rules as above;
+ *   grad_in may equal grad_out and must not overlap x.
+ *   n * element size must not exceed NFAD_NOALLOC_SCRATCH_BYTES (2 097 152 fp32 or
+ *   4 194 304 bf16/fp16 elements); larger calls return NFAD_E_TOO_LARGE and launch
+ *   nothing -- use nfad_cmp_recompute_backward with your own scratch instead.
+ *
+ * The first call on each device looks up the array's device address (a one-time
+ * set-up with that device current); make that first call outside any stream
+ * capture.  All calls on a device share the one array: it still holds whatever
+ * the previous call left there (nothing in it needs to start at zero -- the first
+ * kernel overwrites every byte the second one reads), and two calls whose
+ * kernels may overlap on the GPU (different streams without an ordering between
+ * them) race on it.  Serialise such calls, or give them their own scratch through
+ * nfad_cmp_recompute_backward.
+ */
+#define NFAD_NOALLOC_SCRATCH_BYTES 8388608
+NFAD_API int nfad_cmp_recompute_backward_noalloc(int kind, int dtype, const void* grad_out, const void* x,
+                                                 void* grad_in, size_t n, nfad_stream_t stream);
 
 /* Bytes of scratch the recomputation comparator needs for n elements; 0 on a bad kind or dtype. */
 NFAD_API size_t nfad_cmp_recompute_scratch_bytes(int kind, int dtype, size_t n);

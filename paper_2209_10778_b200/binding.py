@@ -28,8 +28,9 @@ EXPORTS = (
     "nfad_act_forward", "nfad_act_forward_infer", "nfad_act_backward",
     "nfad_cmp_conv_backward", "nfad_cmp_recompute_backward", "nfad_cmp_recompute_scratch_bytes",
     "nfad_saved_bytes_per_element", "nfad_last_cuda_error", "nfad_status_string", "nfad_version",
-    "nfad_probe_stream",
+    "nfad_probe_stream", "nfad_cmp_recompute_backward_noalloc",
 )
+NOALLOC_SCRATCH_BYTES = 8388608
 
 _lib: Optional[ctypes.CDLL] = None
 
@@ -59,6 +60,8 @@ def load() -> ctypes.CDLL:
         lib.nfad_act_backward.argtypes = [ci, ci, vp, vp, vp, sz, vp]
         lib.nfad_cmp_conv_backward.argtypes = [ci, ci, vp, vp, vp, sz, vp]
         lib.nfad_cmp_recompute_backward.argtypes = [ci, ci, vp, vp, vp, sz, vp, sz, vp]
+        lib.nfad_cmp_recompute_backward_noalloc.argtypes = [ci, ci, vp, vp, vp, sz, vp]
+        lib.nfad_cmp_recompute_backward_noalloc.restype = ci
         lib.nfad_cmp_recompute_scratch_bytes.argtypes = [ci, ci, sz]
         lib.nfad_cmp_recompute_scratch_bytes.restype = sz
         lib.nfad_saved_bytes_per_element.argtypes = [ci, ci, ci]
@@ -149,6 +152,18 @@ def nfad_cmp_recompute_backward(kind, grad_out: torch.Tensor, x: torch.Tensor, s
                                                   scratch.data_ptr(), scratch.numel() * scratch.element_size(),
                                                   _tensor(grad_in, "grad_in", grad_out), grad_out.numel(),
                                                   _stream(grad_out)), "nfad_cmp_recompute_backward")
+
+
+def nfad_cmp_recompute_backward_noalloc(kind, grad_out: torch.Tensor, x: torch.Tensor, grad_in: torch.Tensor) -> None:
+    """The recomputation comparator on the library's own fixed scratch array: for callers that
+    cannot allocate device memory where they stand.  At most NOALLOC_SCRATCH_BYTES per tensor;
+    calls on one device share the array, so calls that may overlap on the GPU must be serialised."""
+    pg = _tensor(grad_out, "grad_out")
+    with torch.cuda.device(grad_out.device):
+        _check(load().nfad_cmp_recompute_backward_noalloc(_kind(kind), _TORCH_TO_CODE[grad_out.dtype], pg,
+                                                          _tensor(x, "x", grad_out), _tensor(grad_in, "grad_in", grad_out),
+                                                          grad_out.numel(), _stream(grad_out)),
+               "nfad_cmp_recompute_backward_noalloc")
 
 
 def nfad_saved_bytes_per_element(kind, dtype, layout) -> int:

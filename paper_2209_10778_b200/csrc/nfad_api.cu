@@ -2,6 +2,8 @@
 // and dispatch to the per-storage-type launchers.  No arithmetic lives here.
 #include <stdint.h>
 
+#include <mutex>
+
 #include "../../include/nfad.h"
 #include "nfad_internal.h"
 
@@ -70,6 +72,36 @@ int op_by_op_tensors(int kind)
     case NFAD_GELU_TANH: return 4;
     default: return 3;
     }
+}
+
+// ---- built-in scratch for nfad_cmp_recompute_backward_noalloc ----------------------------
+//
+// The array below lives in the library image: loading the library on a GPU reserves it
+// there until the process exits.  In HOST code the name `g_noalloc_scratch` is only a
+// handle for the runtime, not an address a kernel can use; the device address has to be
+// asked for, once per device, with that device current.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[NFAD_NOALLOC_SCRATCH_BYTES];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_noalloc_mutex;
+void* g_noalloc_ptr[kMaxDevices] = {};
+
+// Device address of the built-in scratch on the current device; looked up on first use.
+cudaError_t noalloc_scratch(void** out)
+{
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+    if (!g_noalloc_ptr[dev]) {
+        void* p = nullptr;
+        e = cudaGetSymbolAddress(&p, g_noalloc_scratch);
+        if (e != cudaSuccess) return e;
+        g_noalloc_ptr[dev] = p;
+    }
+    *out = g_noalloc_ptr[dev];
+    return cudaSuccess;
 }
 
 }  // namespace
@@ -158,6 +190,23 @@ int nfad_probe_stream(int reads, int writes, const void* a, const void* b, void*
     return rc ? rc : run(op, 0, NFAD_F32, in, out, n_words, stream);
 }
 
+int nfad_cmp_recompute_backward_noalloc(int kind, int dtype, const void* grad_out, const void* x, void* grad_in,
+                                        size_t n, nfad_stream_t stream)
+{
+    if (kind < 0 || kind > 3) return NFAD_E_KIND;
+    if (dtype < 0 || dtype > 2) return NFAD_E_DTYPE;
+    if (n == 0) return NFAD_OK;
+    if (n > NFAD_NOALLOC_SCRATCH_BYTES / elem_size(dtype)) return NFAD_E_TOO_LARGE;
+    void* scratch = nullptr;
+    cudaError_t e = noalloc_scratch(&scratch);
+    if (e != cudaSuccess) {
+        g_last_cuda_error = static_cast<int>(e);
+        return NFAD_E_CUDA;
+    }
+    // from here on exactly the two launches of nfad_cmp_recompute_backward, on the built-in array
+    return nfad_cmp_recompute_backward(kind, dtype, grad_out, x, scratch, NFAD_NOALLOC_SCRATCH_BYTES, grad_in, n, stream);
+}
+
 int nfad_saved_bytes_per_element(int kind, int dtype, int layout)
 {
     if (kind < 0 || kind > 3) return -NFAD_E_KIND;
@@ -186,6 +235,7 @@ const char* nfad_status_string(int status)
     case NFAD_E_ALIGN: return "pointer not aligned to the element size";
     case NFAD_E_SCRATCH: return "scratch buffer too small";
     case NFAD_E_LAYOUT: return "unknown layout";
+    case NFAD_E_TOO_LARGE: return "tensors larger than the library's built-in scratch";
     default: return "unknown status";
     }
 }
