@@ -30,6 +30,9 @@ constexpr int kUnroll = NFAD_UNROLL;
 // are issue-bound with short dependency chains through MUFU: 5 CTAs (40 warps, <= 48 registers)
 // measured 3-5 % faster than the 4 the compiler picks by itself (7 or more spill and lose 30 %); the fp32 kernels need their
 // ~48 registers (a tighter cap spills).
+#ifndef NFAD_PDL
+#define NFAD_PDL 1
+#endif
 #ifndef NFAD_MIN_BLOCKS_16
 #define NFAD_MIN_BLOCKS_16 5
 #endif
@@ -136,6 +139,7 @@ template <int NIN, int NOUT> struct StreamArgs {
 // Op: struct with
 //   static constexpr int kIn, kOut;  static constexpr bool keep(int out_slot);
 //   static __device__ void apply(const float (&in)[kIn], float (&out)[kOut]);
+//   static constexpr int kMinBlocks: resident CTAs per SM to leave room for (0: the storage type's default);
 //   static constexpr bool kPacketFixup; if set, fixup(vin, vout) may patch a whole packet's
 //   results after apply (a rare case kept off the per-element path) and apply_checked is the
 //   one-element form that includes the patch.
@@ -182,12 +186,22 @@ __device__ __forceinline__ void packet_compute_store(const StreamArgs<Op::kIn, O
 }
 
 template <class S, class Op>
-__global__ void __launch_bounds__(kBlock, S::kMinBlocks) stream_kernel(const StreamArgs<Op::kIn, Op::kOut> a)
+__global__ void __launch_bounds__(kBlock, (Op::kMinBlocks ? Op::kMinBlocks : S::kMinBlocks)) stream_kernel(const StreamArgs<Op::kIn, Op::kOut> a)
 {
     constexpr int V = S::kVec;
     const size_t byte_off = a.head * sizeof(typename S::elem);
     const size_t tile_packets = size_t(kBlock) * kUnroll;
     const size_t n_tiles = (a.packets + tile_packets - 1) / tile_packets;
+
+#if NFAD_PDL
+    // Programmatic dependent launch: let the next kernel of the stream be scheduled onto SMs
+    // as this grid's last CTAs drain (it is only released once every CTA of this grid has
+    // started), and do not touch memory before the previous kernel of the stream has
+    // completed and its writes are visible.  Both are no-ops for a launch without the
+    // programmatic-serialisation attribute.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+#endif
 
     for (size_t tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
         const size_t base = tile * tile_packets + threadIdx.x;
@@ -307,8 +321,22 @@ cudaError_t launch_stream(const void* const* in, void* const* out, size_t n, cud
     // the tiles (the window of addresses in flight stays compact), and it balances the SMs at
     // tile granularity.  The kernel's tile loop only matters beyond 2^31-1 tiles.
     size_t grid = tiles < size_t(0x7fffffff) ? tiles : size_t(0x7fffffff);
+#if NFAD_PDL
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3(kBlock);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, stream_kernel<S, Op>, a);
+#else
     stream_kernel<S, Op><<<(unsigned)grid, kBlock, 0, st>>>(a);
     return cudaPeekAtLastError();
+#endif
 }
 
 }  // namespace nfad
