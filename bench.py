@@ -186,7 +186,7 @@ def run_reference(args, w):
 
 def run_ours(args, w):
     import torch
-    import torch.distributed as dist
+    from paper_2209_10778_b200 import ranks
     from paper_2209_10778_b200 import binding as nfad
     from paper_2209_10778_b200 import workloads as W
 
@@ -194,13 +194,11 @@ def run_ours(args, w):
         raise RuntimeError("bench.py needs a CUDA device: the path has no CPU implementation")
     nfad.load()                                    # fails loudly if libnfad.so is missing
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    wd = ranks.world_from_env()
+    world, rank, local_rank = wd.size, wd.rank, wd.local_rank
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=dev)
+    ranks.init(wd, "nccl", dev)
 
     n = w.numel(0)
     es = 4 if w.dtype == "f32" else 2
@@ -276,9 +274,7 @@ def run_ours(args, w):
             count -= 1
 
     def barrier():
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
+        ranks.barrier(wd, cuda=True)
 
     sampler = ClockSampler(local_rank) if rank == 0 else None
     if sampler:
@@ -306,10 +302,7 @@ def run_ours(args, w):
         t_wall1 = time.time()
     if sampler:
         sampler.stop()
-    if world > 1:
-        t = torch.tensor([ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = ranks.max_over_ranks(wd, ms, dev)
 
     timing_source = "events around single launches at the end of the timed region"
     src = ev
@@ -346,19 +339,15 @@ def run_ours(args, w):
     s1.record()
     barrier()
     e2e_ms = s0.elapsed_time(s1)
-    if world > 1:
-        t = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
+    e2e_ms = ranks.max_over_ranks(wd, e2e_ms, dev)
 
     if rank != 0:
-        if world > 1:
-            dist.destroy_process_group()
+        ranks.finish(wd)
         return
 
     elems_per_step = n * len(kinds)
-    value = world * elems_per_step * args.steps / (ms / 1e3)
-    e2e_value = world * elems_per_step * e2e_steps / (e2e_ms / 1e3)
+    value = ranks.whole_job_rate(wd, elems_per_step, args.steps, ms)
+    e2e_value = ranks.whole_job_rate(wd, elems_per_step, e2e_steps, e2e_ms)
     peak, peak_kind = _peaks()
     algo_bytes = 3 * es * n                       # forward: read x, write y and f'
     achieved = algo_bytes / (fwd_ms / 1e3) / 1e9 if fwd_ms else None
@@ -421,8 +410,7 @@ def run_ours(args, w):
         "clocks": sampler.summary(t_wall0, t_wall1, window) if sampler else None,
     }
     print(json.dumps(line), flush=True)
-    if world > 1:
-        dist.destroy_process_group()
+    ranks.finish(wd)
 
 
 def main():
