@@ -71,7 +71,8 @@ typedef enum {
     NFAD_E_ALIGN = 6,    /* a pointer is not a multiple of the element size           */
     NFAD_E_SCRATCH = 7,  /* scratch_bytes is smaller than the comparator needs        */
     NFAD_E_LAYOUT = 8,   /* layout is not an nfad_layout                              */
-    NFAD_E_TOO_LARGE = 9 /* the tensors need more than the library's built-in scratch */
+    NFAD_E_TOO_LARGE = 9, /* the tensors need more than the library's built-in scratch */
+    NFAD_E_PROGRAM = 10  /* malformed FAD sequence (see nfad_seq_forward)              */
 } nfad_status;
 
 /* How the tensor needed by backward is kept between the passes (Section II-C). */
@@ -181,6 +182,66 @@ NFAD_API size_t nfad_cmp_recompute_scratch_bytes(int kind, int dtype, size_t n);
  * Returns a negative nfad_status on a bad argument.
  */
 NFAD_API int nfad_saved_bytes_per_element(int kind, int dtype, int layout);
+
+/*
+ * FAD sequences composed at run time.
+ *
+ * The paper's method is not tied to four activations: any run of FAD-compatible
+ * primitive operations (Section III-A: unary operations, binary operations whose
+ * two inputs come from the same source, binary operations with one constant)
+ * with one source and M >= 1 results (R^1 -> R^M, Section II-D "Computation
+ * efficiency" and the state sequence NY, YY.., YN of Section IV) can be nested in
+ * back-propagation the same way.  A sequence is a straight-line program over 12
+ * dual registers; register 0 holds the source (x, tangent 1).  Each instruction
+ * applies one primitive to register a (and b for ADD / MUL, which merge two
+ * branches of the same source) and writes register dst; NFAD_OP_OUT copies
+ * register a to result slot dst (0 <= dst < m).  SCALE and ADD_CONST take their
+ * constant from c.
+ *
+ *   program [host] n_ops <= 32 instructions.  Malformed programs (unknown opcode, register
+ *           out of range, a register read before it is written, a result slot out of
+ *           range or never written) give NFAD_E_PROGRAM.
+ *   x       [in]   n elements.
+ *   y, dfdx [host arrays of m device pointers, m <= 4] y[k][i] = k-th result, dfdx[k][i] its
+ *           derivative with respect to x[i]: per result, the one tensor to keep.
+ * One kernel runs the whole sequence per element on dual numbers; no intermediate reaches
+ * memory.  Arithmetic: plain fp32 primitives for every storage type (a few fp32 ulp where
+ * the composed function is well conditioned) -- the four activations of Table I have
+ * dedicated, hardened entry points above.  Outputs must not overlap each other or x.
+ */
+typedef enum {
+    NFAD_OP_ADD = 0, NFAD_OP_MUL = 1, NFAD_OP_SCALE = 2, NFAD_OP_ADD_CONST = 3, NFAD_OP_EXP = 4, NFAD_OP_LOG1P = 5,
+    NFAD_OP_TANH = 6, NFAD_OP_ERF = 7, NFAD_OP_SOFTPLUS = 8, NFAD_OP_SIGMOID = 9, NFAD_OP_HALF_ONE_PLUS_TANH = 10,
+    NFAD_OP_HALF_ONE_PLUS_ERF = 11, NFAD_OP_OUT = 12
+} nfad_opcode;
+
+typedef struct { int op; int a; int b; int dst; float c; } nfad_seq_op;
+
+NFAD_API int nfad_seq_forward(const nfad_seq_op* program, int n_ops, int dtype, const void* x, void* const* y,
+                              void* const* dfdx, int m, size_t n, nfad_stream_t stream);
+
+/*
+ * Backward of a sequence with m results (Section II-E; for a binary merge "the post-process
+ * will merge (accumulate) FAD results", Section IV): grad_in[i] = sum_k grad_out[k][i] * dfdx[k][i],
+ * accumulated in fp32 in the order k = 0..m-1 with fused multiply-adds and rounded once.
+ * For m == 1 this is nfad_act_backward.  grad_out, dfdx: host arrays of m device pointers.
+ */
+NFAD_API int nfad_seq_backward(int dtype, const void* const* grad_out, const void* const* dfdx, int m, void* grad_in,
+                               size_t n, nfad_stream_t stream);
+
+/*
+ * One primitive as its own kernel, the way a framework runs it when every operator is a node
+ * of the graph (Section II-C approach 1); used to MEASURE operator-by-operator back-propagation.
+ *   forward  (backward == 0): out0 = op(in0 [, in1]) for ADD / MUL, op(in0) otherwise.
+ *   backward (backward != 0): in0 = upstream gradient; in1 (, in2) = what the operator's rule kept:
+ *       MUL: both operands (out0 = g * in2 is the gradient of the first operand, out1 = g * in1 of the second);
+ *       EXP, TANH, SIGMOID, HALF_ONE_PLUS_TANH: the forward output;
+ *       LOG1P, ERF, SOFTPLUS, HALF_ONE_PLUS_ERF: the forward input;  SCALE: nothing.
+ *       ADD and ADD_CONST pass the gradient through and need no kernel.
+ * Unused pointers are NULL.  Exact in-place use allowed.
+ */
+NFAD_API int nfad_ew_op(int op, int backward, float c, int dtype, const void* in0, const void* in1, const void* in2,
+                        void* out0, void* out1, size_t n, nfad_stream_t stream);
 
 /*
  * Traffic probe (a measurement aid with no counterpart in the paper): moves

@@ -25,6 +25,7 @@ DTYPES = {"f32": 0, "bf16": 1, "f16": 2}
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "nfad_oracle.c")
+_SRC_SEQ = os.path.join(_HERE, "nfad_seq_oracle.c")
 _LIB = os.path.join(_HERE, "libnfad_oracle.so")
 _lock = threading.Lock()
 _lib = None
@@ -33,10 +34,10 @@ _lib = None
 def build(force: bool = False) -> str:
     """Compile the oracle with gcc (IEEE semantics: no fast-math, no contraction)."""
     with _lock:
-        stale = (not os.path.exists(_LIB)) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC)
+        stale = (not os.path.exists(_LIB)) or os.path.getmtime(_LIB) < max(os.path.getmtime(_SRC), os.path.getmtime(_SRC_SEQ))
         if force or stale:
             cmd = ["gcc", "-O2", "-std=c11", "-fPIC", "-shared", "-fopenmp",
-                   "-ffp-contract=off", "-fno-fast-math", "-o", _LIB, _SRC, "-lm"]
+                   "-ffp-contract=off", "-fno-fast-math", "-o", _LIB, _SRC, _SRC_SEQ, "-lm"]
             subprocess.run(cmd, check=True, capture_output=True)
     return _LIB
 
@@ -63,6 +64,11 @@ def _load():
                      "nfad_oracle_get_threads", "nfad_oracle_max_threads"):
             getattr(lib, name).restype = ci
         lib.nfad_oracle_set_threads.restype = None
+        ip, dp = ctypes.POINTER(ctypes.c_int), ctypes.POINTER(ctypes.c_double)
+        lib.nfad_seq_oracle_forward.argtypes = [ci, ip, ip, ip, ip, dp, vp, sz, ci, vp, vp]
+        lib.nfad_seq_oracle_forward.restype = ci
+        lib.nfad_seq_oracle_backward.argtypes = [vp, vp, sz, ci, vp, vp]
+        lib.nfad_seq_oracle_backward.restype = ci
         _lib = lib
     return _lib
 
@@ -164,3 +170,35 @@ def forward_backward(kind, dtype, x: np.ndarray, grad_out: np.ndarray):
     _ok(_load().nfad_oracle_forward_backward(_code(KINDS, kind), _code(DTYPES, dtype), _ptr(x), _ptr(g),
                                              x.size, _ptr(y), _ptr(d), _ptr(gin)), "forward_backward")
     return y, d, gin
+
+
+SEQ_OPCODES = {"add": 0, "mul": 1, "scale": 2, "add_const": 3, "exp": 4, "log1p": 5, "tanh": 6, "erf": 7, "softplus": 8,
+               "sigmoid": 9, "half_one_plus_tanh": 10, "half_one_plus_erf": 11, "out": 12}
+
+
+def seq_forward(program, x: np.ndarray, m: int):
+    """A FAD sequence in fp64.  program: list of (op name, a, b, dst, c); x: fp64 array.
+    Returns (y, dydx), each of shape (m, n)."""
+    n_ops = len(program)
+    IntArr, DblArr = ctypes.c_int * n_ops, ctypes.c_double * n_ops
+    op = IntArr(*[SEQ_OPCODES[o[0]] for o in program])
+    a = IntArr(*[int(o[1]) for o in program])
+    b = IntArr(*[int(o[2]) for o in program])
+    dst = IntArr(*[int(o[3]) for o in program])
+    c = DblArr(*[float(o[4]) for o in program])
+    x = np.ascontiguousarray(x, np.float64).reshape(-1)
+    y = np.empty((m, x.size), np.float64)
+    d = np.empty((m, x.size), np.float64)
+    _ok(_load().nfad_seq_oracle_forward(n_ops, op, a, b, dst, c, _ptr(x), x.size, m, _ptr(y), _ptr(d)), "seq_forward")
+    return y, d
+
+
+def seq_backward(g: np.ndarray, d: np.ndarray):
+    """(sum_k g_k d_k, sum_k |g_k d_k|) in fp64 for operands of shape (m, n)."""
+    g = np.ascontiguousarray(g, np.float64)
+    d = np.ascontiguousarray(d, np.float64)
+    m, n = g.shape
+    out = np.empty(n, np.float64)
+    out_abs = np.empty(n, np.float64)
+    _ok(_load().nfad_seq_oracle_backward(_ptr(g), _ptr(d), n, m, _ptr(out), _ptr(out_abs)), "seq_backward")
+    return out, out_abs

@@ -9,5 +9,6 @@ from .binding import (  # noqa: F401
     nfad_act_backward, nfad_act_forward, nfad_act_forward_infer,
     nfad_cmp_conv_backward, nfad_cmp_recompute_backward, nfad_cmp_recompute_backward_noalloc,
     nfad_cmp_recompute_scratch_bytes,
-    nfad_probe_stream, nfad_saved_bytes_per_element, nfad_status_string, nfad_version,
+    nfad_ew_op, nfad_probe_stream, nfad_saved_bytes_per_element, nfad_seq_backward, nfad_seq_forward,
+    nfad_status_string, nfad_version,
 )

@@ -29,7 +29,15 @@ EXPORTS = (
     "nfad_cmp_conv_backward", "nfad_cmp_recompute_backward", "nfad_cmp_recompute_scratch_bytes",
     "nfad_saved_bytes_per_element", "nfad_last_cuda_error", "nfad_status_string", "nfad_version",
     "nfad_probe_stream", "nfad_cmp_recompute_backward_noalloc",
+    "nfad_seq_forward", "nfad_seq_backward", "nfad_ew_op",
 )
+OPCODES = {"add": 0, "mul": 1, "scale": 2, "add_const": 3, "exp": 4, "log1p": 5, "tanh": 6, "erf": 7, "softplus": 8,
+           "sigmoid": 9, "half_one_plus_tanh": 10, "half_one_plus_erf": 11, "out": 12}
+
+
+class SeqOp(ctypes.Structure):
+    """One instruction of a FAD sequence: `nfad_seq_op` of the C interface."""
+    _fields_ = [("op", ctypes.c_int), ("a", ctypes.c_int), ("b", ctypes.c_int), ("dst", ctypes.c_int), ("c", ctypes.c_float)]
 NOALLOC_SCRATCH_BYTES = 8388608
 
 _lib: Optional[ctypes.CDLL] = None
@@ -62,6 +70,12 @@ def load() -> ctypes.CDLL:
         lib.nfad_cmp_recompute_backward.argtypes = [ci, ci, vp, vp, vp, sz, vp, sz, vp]
         lib.nfad_cmp_recompute_backward_noalloc.argtypes = [ci, ci, vp, vp, vp, sz, vp]
         lib.nfad_cmp_recompute_backward_noalloc.restype = ci
+        lib.nfad_seq_forward.argtypes = [ctypes.POINTER(SeqOp), ci, ci, vp, ctypes.POINTER(vp), ctypes.POINTER(vp), ci, sz, vp]
+        lib.nfad_seq_forward.restype = ci
+        lib.nfad_seq_backward.argtypes = [ci, ctypes.POINTER(vp), ctypes.POINTER(vp), ci, vp, sz, vp]
+        lib.nfad_seq_backward.restype = ci
+        lib.nfad_ew_op.argtypes = [ci, ci, ctypes.c_float, ci, vp, vp, vp, vp, vp, sz, vp]
+        lib.nfad_ew_op.restype = ci
         lib.nfad_cmp_recompute_scratch_bytes.argtypes = [ci, ci, sz]
         lib.nfad_cmp_recompute_scratch_bytes.restype = sz
         lib.nfad_saved_bytes_per_element.argtypes = [ci, ci, ci]
@@ -164,6 +178,53 @@ def nfad_cmp_recompute_backward_noalloc(kind, grad_out: torch.Tensor, x: torch.T
                                                           _tensor(x, "x", grad_out), _tensor(grad_in, "grad_in", grad_out),
                                                           grad_out.numel(), _stream(grad_out)),
                "nfad_cmp_recompute_backward_noalloc")
+
+
+def _ptr_array(tensors, name, like):
+    arr = (ctypes.c_void_p * len(tensors))()
+    for i, t in enumerate(tensors):
+        arr[i] = _tensor(t, f"{name}[{i}]", like)
+    return arr
+
+
+def nfad_seq_forward(program, x: torch.Tensor, ys, dfdxs) -> None:
+    """Runs a FAD sequence (a list of SeqOp, or of (op, a, b, dst, c) tuples with op a name or code)
+    on x in one kernel: ys[k] = k-th result, dfdxs[k] = its derivative with respect to x."""
+    ops = (SeqOp * len(program))()
+    for i, o in enumerate(program):
+        if isinstance(o, SeqOp):
+            ops[i] = o
+        else:
+            op, a, b, dst, c = o
+            ops[i] = SeqOp(OPCODES[op] if isinstance(op, str) else int(op), int(a), int(b), int(dst), float(c))
+    px = _tensor(x, "x")
+    if len(ys) != len(dfdxs):
+        raise ValueError("ys and dfdxs must have the same length")
+    with torch.cuda.device(x.device):
+        _check(load().nfad_seq_forward(ops, len(program), _TORCH_TO_CODE[x.dtype], px, _ptr_array(ys, "y", x),
+                                       _ptr_array(dfdxs, "dfdx", x), len(ys), x.numel(), _stream(x)), "nfad_seq_forward")
+
+
+def nfad_seq_backward(grad_outs, dfdxs, grad_in: torch.Tensor) -> None:
+    """grad_in = sum_k grad_outs[k] * dfdxs[k]."""
+    pg = _tensor(grad_in, "grad_in")
+    if len(grad_outs) != len(dfdxs):
+        raise ValueError("grad_outs and dfdxs must have the same length")
+    with torch.cuda.device(grad_in.device):
+        _check(load().nfad_seq_backward(_TORCH_TO_CODE[grad_in.dtype], _ptr_array(grad_outs, "grad_out", grad_in),
+                                        _ptr_array(dfdxs, "dfdx", grad_in), len(grad_outs), pg, grad_in.numel(),
+                                        _stream(grad_in)), "nfad_seq_backward")
+
+
+def nfad_ew_op(op, backward: bool, c: float, in0: torch.Tensor, in1, in2, out0: torch.Tensor, out1=None) -> None:
+    """One primitive as its own kernel (forward, or its own backward rule): see include/nfad.h."""
+    p0 = _tensor(in0, "in0")
+    code = OPCODES[op] if isinstance(op, str) else int(op)
+    opt = lambda t, name: _tensor(t, name, in0) if t is not None else None
+    with torch.cuda.device(in0.device):
+        _check(load().nfad_ew_op(code, 1 if backward else 0, float(c), _TORCH_TO_CODE[in0.dtype], p0, opt(in1, "in1"),
+                                 opt(in2, "in2"), _tensor(out0, "out0", in0), opt(out1, "out1"), in0.numel(), _stream(in0)),
+               "nfad_ew_op")
 
 
 def nfad_saved_bytes_per_element(kind, dtype, layout) -> int:

@@ -27,6 +27,7 @@ COMMON = ["-O3", "-std=c++17", "-lineinfo", "-Xcompiler", "-fPIC", "-Xcompiler",
 UNITS = [
     ("nfad_kernels_f32.cu", ["-fmad=false"]),
     ("nfad_kernels_16.cu", ["-fmad=true"]),
+    ("nfad_kernels_seq.cu", ["-fmad=true"]),
     ("nfad_api.cu", ["-fmad=false"]),
 ]
 

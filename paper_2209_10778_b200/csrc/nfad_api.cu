@@ -207,6 +207,86 @@ int nfad_cmp_recompute_backward_noalloc(int kind, int dtype, const void* grad_ou
     return nfad_cmp_recompute_backward(kind, dtype, grad_out, x, scratch, NFAD_NOALLOC_SCRATCH_BYTES, grad_in, n, stream);
 }
 
+int nfad_seq_forward(const nfad_seq_op* program, int n_ops, int dtype, const void* x, void* const* y, void* const* dfdx,
+                     int m, size_t n, nfad_stream_t stream)
+{
+    if (dtype < 0 || dtype > 2) return NFAD_E_DTYPE;
+    if (!program || !y || !dfdx) return NFAD_E_NULL;
+    if (n_ops < 1 || n_ops > nfad::kSeqMaxOpsHost || m < 1 || m > 4) return NFAD_E_PROGRAM;
+    nfad::SeqProgramHost p;
+    p.n_ops = n_ops;
+    constexpr int kRegs = 12;
+    bool written[kRegs] = {true};
+    bool produced[4] = {false, false, false, false};
+    for (int i = 0; i < n_ops; ++i) {
+        const nfad_seq_op& o = program[i];
+        if (o.op < 0 || o.op > NFAD_OP_OUT) return NFAD_E_PROGRAM;
+        if (o.a < 0 || o.a >= kRegs || !written[o.a]) return NFAD_E_PROGRAM;
+        const bool binary = o.op == NFAD_OP_ADD || o.op == NFAD_OP_MUL;
+        if (binary && (o.b < 0 || o.b >= kRegs || !written[o.b])) return NFAD_E_PROGRAM;
+        if (o.op == NFAD_OP_OUT) {
+            if (o.dst < 0 || o.dst >= m) return NFAD_E_PROGRAM;
+            produced[o.dst] = true;
+        } else {
+            if (o.dst < 1 || o.dst >= kRegs) return NFAD_E_PROGRAM;  // register 0 is the source and stays it
+            written[o.dst] = true;
+        }
+        p.op[i] = o.op; p.a[i] = o.a; p.b[i] = binary ? o.b : o.a; p.dst[i] = o.dst; p.c[i] = o.c;
+    }
+    for (int k = 0; k < m; ++k) if (!produced[k]) return NFAD_E_PROGRAM;
+    const void* in[1] = {x};
+    void* out[8];
+    for (int k = 0; k < m; ++k) { out[k] = y[k]; out[m + k] = dfdx[k]; }
+    int rc = check(0, dtype, in, 1, out, 2 * m, n);
+    if (rc) return rc;
+    if (n == 0) return NFAD_OK;
+    for (int k = 0; k < 2 * m; ++k) if (out[k] == x) return NFAD_E_OVERLAP;
+    cudaError_t e = nfad::launch_seq_forward(p, dtype, x, y, dfdx, m, n, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) { g_last_cuda_error = static_cast<int>(e); return NFAD_E_CUDA; }
+    return NFAD_OK;
+}
+
+int nfad_seq_backward(int dtype, const void* const* grad_out, const void* const* dfdx, int m, void* grad_in, size_t n,
+                      nfad_stream_t stream)
+{
+    if (dtype < 0 || dtype > 2) return NFAD_E_DTYPE;
+    if (!grad_out || !dfdx) return NFAD_E_NULL;
+    if (m < 1 || m > 4) return NFAD_E_PROGRAM;
+    const void* in[8];
+    for (int k = 0; k < m; ++k) { in[k] = grad_out[k]; in[m + k] = dfdx[k]; }
+    void* out[1] = {grad_in};
+    int rc = check(0, dtype, in, 2 * m, out, 1, n);
+    if (rc) return rc;
+    if (n == 0) return NFAD_OK;
+    cudaError_t e = nfad::launch_seq_backward(dtype, grad_out, dfdx, m, grad_in, n, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) { g_last_cuda_error = static_cast<int>(e); return NFAD_E_CUDA; }
+    return NFAD_OK;
+}
+
+int nfad_ew_op(int op, int backward, float c, int dtype, const void* in0, const void* in1, const void* in2, void* out0,
+               void* out1, size_t n, nfad_stream_t stream)
+{
+    if (dtype < 0 || dtype > 2) return NFAD_E_DTYPE;
+    if (op < 0 || op >= NFAD_OP_OUT) return NFAD_E_PROGRAM;
+    const void* in[3];
+    int nin = 0;
+    in[nin++] = in0;
+    if (in1) in[nin++] = in1;
+    if (in2) in[nin++] = in2;
+    void* out[2];
+    int nout = 0;
+    out[nout++] = out0;
+    if (out1) out[nout++] = out1;
+    int rc = check(0, dtype, in, nin, out, nout, n);
+    if (rc) return rc;
+    if (n == 0) return NFAD_OK;
+    const void* in3[3] = {in0, in1, in2};
+    void* out2[2] = {out0, out1};
+    cudaError_t e = nfad::launch_ew(op, backward ? 1 : 0, c, dtype, in3, out2, n, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) { g_last_cuda_error = static_cast<int>(e); return NFAD_E_CUDA; }
+    return NFAD_OK;
+}
+
 int nfad_saved_bytes_per_element(int kind, int dtype, int layout)
 {
     if (kind < 0 || kind > 3) return -NFAD_E_KIND;
@@ -236,6 +316,7 @@ const char* nfad_status_string(int status)
     case NFAD_E_SCRATCH: return "scratch buffer too small";
     case NFAD_E_LAYOUT: return "unknown layout";
     case NFAD_E_TOO_LARGE: return "tensors larger than the library's built-in scratch";
+    case NFAD_E_PROGRAM: return "malformed FAD sequence";
     default: return "unknown status";
     }
 }

@@ -14,7 +14,7 @@
 // the closed symbolic forms tanh / sigmoid / softplus that frameworks ship as
 // single operators):
 //     dual_add  dual_mul  dual_scale  dual_add_const
-//     dual_tanh  dual_softplus  dual_sigmoid
+//     dual_exp  dual_log1p  dual_tanh  dual_erf  dual_softplus  dual_sigmoid
 // and two "binary with a constant, hence unary" fusions that keep the tails
 // free of cancellation:
 //     dual_half_one_plus_tanh(u) = (1 + tanh u)/2 = sigmoid(2u)
@@ -295,6 +295,69 @@ NFAD_DEV Gate<Full> dual_tanh(const SoftplusDual<Full>& p)
     float tt = f2_value(f2_mul(a1, rd2)) * (neg ? 4.0f : 4.0f * e.h);
     F2 v = neg ? sm : F2{1.0f, -f2_value(sm)};
     return {v, tt, neg ? sc : 1.0f, neg ? p.E.n : 0};
+}
+
+// ----------------------------------------------------------------- general-purpose primitives (Fast policy)
+//
+// exp, log1p, tanh, erf and the value of softplus are not needed by the four
+// activation chains above (which use the cancellation-free fusions); they are the
+// remaining members of the primitive set, for sequences composed at run time.
+// Plain fp32 on MUFU ex2 / lg2 / rcp: good to a few fp32 ulp of the value where the
+// function itself is well conditioned; a user who writes 1 + tanh(u) gets the
+// cancellation that expression has.
+
+// exp:  v = e^a,  v' = v
+NFAD_DEV Dual<Fast> dual_exp(const Dual<Fast>& a)
+{
+    float v = hw::ex2_approx(1.44269502f * a.v);
+    return {v, v * a.t};
+}
+
+// log1p:  v = log(1 + a),  v' = 1/(1 + a).  log(u) a/(u - 1) with u = fl(1 + a) cancels
+// the rounding of u to first order; a itself when u rounds to 1.
+NFAD_DEV Dual<Fast> dual_log1p(const Dual<Fast>& a)
+{
+    float u = 1.0f + a.v;
+    float lg = 0.693147182f * hw::lg2_approx(u);
+    float um1 = u - 1.0f;
+    float v = um1 == 0.0f ? a.v : lg * (a.v * hw::rcp_approx(um1));
+    return {v, a.t * hw::rcp_approx(u)};
+}
+
+// tanh:  v' = 1 - v^2, formed as 4e/(1+e)^2 from e = exp(-2|a|) so that it stays
+// accurate where v -> 1; an odd polynomial takes over for small |a|, where (1-e)/(1+e) cancels.
+NFAD_DEV Dual<Fast> dual_tanh(const Dual<Fast>& a)
+{
+    float aa = fabsf(a.v);
+    float e = hw::ex2_approx(-2.88539004f * aa);
+    float r = hw::rcp_approx(1.0f + e);
+    float big = (1.0f - e) * r;
+    float a2 = a.v * a.v;
+    float small_ = aa * fmaf(a2, fmaf(a2, fmaf(a2, -0.0539682545f, 0.133333340f), -0.333333343f), 1.0f);
+    float v = copysignf(aa < 0.25f ? small_ : big, a.v);
+    float slope = aa < 0.25f ? fmaf(-v, v, 1.0f) : (4.0f * e) * (r * r);
+    return {v, slope * a.t};
+}
+
+// erf:  v' = 2/sqrt(pi) exp(-a^2).  1 - erfc for |a| >= 0.5, the Maclaurin series below.
+NFAD_DEV Dual<Fast> dual_erf(const Dual<Fast>& a)
+{
+    float aa = fabsf(a.v);
+    float a2 = aa * aa;
+    float e64 = exp2_fast_times_2p64(fmaf(a2, -1.44269502f, 64.0f));
+    float big = fmaf(-2.0f, e64 * half_erfcx_fast_scaled(aa), 1.0f);
+    float ser = fmaf(a2, fmaf(a2, fmaf(a2, fmaf(a2, 0.00522397785f, -0.0268661696f), 0.112837918f), -0.376126379f), 1.12837923f);
+    float v = copysignf(aa < 0.5f ? aa * ser : big, a.v);
+    return {v, (e64 * (1.12837923f * kTwoPowMinus64)) * a.t};
+}
+
+// softplus with its value:  v = max(a, 0) + log1p(exp(-|a|)),  v' = sigmoid(a)
+NFAD_DEV Dual<Fast> dual_softplus(const Dual<Fast>& a)
+{
+    float e = exp2_fast_times_2p64(fmaf(fabsf(a.v), -1.44269502f, 64.0f)) * kTwoPowMinus64;
+    Dual<Fast> l = dual_log1p(Dual<Fast>{e, 0.0f});
+    float r = hw::rcp_approx(1.0f + e);
+    return {fmaxf(a.v, 0.0f) + l.v, (a.v < 0.0f ? e * r : r) * a.t};
 }
 
 // ----------------------------------------------------------------- the four activations (Table I)

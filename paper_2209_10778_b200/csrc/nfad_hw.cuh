@@ -36,6 +36,14 @@ NFAD_DEV float clamp_nan(float a, float lo, float hi)
     return r;
 }
 
+// log2(a), MUFU.LG2 (keeps subnormal inputs).
+NFAD_DEV float lg2_approx(float a)
+{
+    float r;
+    asm("lg2.approx.f32 %0, %1;" : "=f"(r) : "f"(a));
+    return r;
+}
+
 // max(a, lo) that returns NaN for a NaN.
 NFAD_DEV float max_nan(float a, float lo)
 {

@@ -25,4 +25,14 @@ enum OpCode { kOpForward, kOpForwardInfer, kOpBackward, kOpConvBackward, kOpReco
 cudaError_t launch_f32(OpCode op, int kind, const void* const* in, void* const* out, size_t n, cudaStream_t st);
 cudaError_t launch_16(OpCode op, int kind, int dtype, const void* const* in, void* const* out, size_t n, cudaStream_t st);
 
+// Run-time FAD sequences (nfad_seq.cuh): the program as plain arrays, so that this header
+// stays free of device code.
+constexpr int kSeqMaxOpsHost = 32;
+struct SeqProgramHost { int n_ops; int op[kSeqMaxOpsHost], a[kSeqMaxOpsHost], b[kSeqMaxOpsHost], dst[kSeqMaxOpsHost]; float c[kSeqMaxOpsHost]; };
+
+cudaError_t launch_seq_forward(const SeqProgramHost& p, int dtype, const void* x, void* const* y, void* const* d, int m, size_t n,
+                               cudaStream_t st);
+cudaError_t launch_seq_backward(int dtype, const void* const* g, const void* const* d, int m, void* gin, size_t n, cudaStream_t st);
+cudaError_t launch_ew(int op, int backward, float c, int dtype, const void* const* in, void* const* out, size_t n, cudaStream_t st);
+
 }  // namespace nfad

@@ -1,0 +1,249 @@
+// nfad_seq.cuh -- FAD sequences composed at run time.
+//
+// A FAD sequence (Section IV: the run of fad operators between the NY and YN
+// states) is a straight-line program over at most kSeqRegs dual registers;
+// register 0 holds the seed (x, 1).  Every instruction is one primitive operation
+// of Section III-A: unary, binary with both inputs from the same source (add, mul:
+// the "merge" of two branches), or binary with a constant.  OUT copies a register
+// to one of m <= kSeqMaxOut outputs: one source, M results (R^1 -> R^M).  One kernel
+// interprets the whole program per element on dual numbers, so no intermediate and
+// no intermediate derivative reaches memory; per output only y_k and dy_k/dx do.
+//
+// The program is the same for every element, so the interpreter's control flow is
+// uniform; registers are indexed at run time and therefore live in local memory.
+// This executor trades speed for generality; the four activations of Table I have
+// the dedicated kernels.
+#pragma once
+
+#include "nfad_dual.cuh"
+#include "nfad_stream.cuh"
+
+namespace nfad {
+
+constexpr int kSeqMaxOps = 32;
+constexpr int kSeqRegs = 12;
+constexpr int kSeqMaxOut = 4;
+
+enum SeqOpcode {
+    kSeqAdd = 0, kSeqMul = 1, kSeqScale = 2, kSeqAddConst = 3, kSeqExp = 4, kSeqLog1p = 5, kSeqTanh = 6, kSeqErf = 7,
+    kSeqSoftplus = 8, kSeqSigmoid = 9, kSeqHalfOnePlusTanh = 10, kSeqHalfOnePlusErf = 11, kSeqOut = 12, kSeqOpcodeCount = 13
+};
+
+struct SeqOp { int op, a, b, dst; float c; };
+struct SeqProgram { int n_ops; SeqOp ops[kSeqMaxOps]; };
+
+// One primitive on duals (Fast policy: plain fp32).
+__device__ __forceinline__ Dual<Fast> seq_apply(const SeqOp& o, const Dual<Fast>& a, const Dual<Fast>& b)
+{
+    switch (o.op) {
+    case kSeqAdd: return dual_add(a, b);
+    case kSeqMul: return dual_mul(a, b);
+    case kSeqScale: return Dual<Fast>{o.c * a.v, o.c * a.t};
+    case kSeqAddConst: return dual_add_const(o.c, a);
+    case kSeqExp: return dual_exp(a);
+    case kSeqLog1p: return dual_log1p(a);
+    case kSeqTanh: return dual_tanh(a);
+    case kSeqErf: return dual_erf(a);
+    case kSeqSoftplus: return dual_softplus(a);
+    case kSeqSigmoid: return as_dual(dual_sigmoid(a));
+    case kSeqHalfOnePlusTanh: return as_dual(dual_half_one_plus_tanh(a));
+    case kSeqHalfOnePlusErf: return as_dual(dual_half_one_plus_erf(a));
+    default: return a;
+    }
+}
+
+template <int V>
+__device__ __forceinline__ void seq_run(const SeqProgram& prog, const float (&x)[V], float (&yv)[kSeqMaxOut][V],
+                                        float (&yt)[kSeqMaxOut][V])
+{
+    float rv[kSeqRegs][V], rt[kSeqRegs][V];
+#pragma unroll
+    for (int e = 0; e < V; ++e) { rv[0][e] = x[e]; rt[0][e] = 1.0f; }
+    for (int i = 0; i < prog.n_ops; ++i) {
+        const SeqOp o = prog.ops[i];
+        if (o.op == kSeqOut) {
+#pragma unroll
+            for (int e = 0; e < V; ++e) { yv[o.dst][e] = rv[o.a][e]; yt[o.dst][e] = rt[o.a][e]; }
+        } else {
+#pragma unroll
+            for (int e = 0; e < V; ++e) {
+                Dual<Fast> r = seq_apply(o, Dual<Fast>{rv[o.a][e], rt[o.a][e]}, Dual<Fast>{rv[o.b][e], rt[o.b][e]});
+                rv[o.dst][e] = r.v;
+                rt[o.dst][e] = r.t;
+            }
+        }
+    }
+}
+
+struct SeqForwardArgs {
+    const void* x;
+    void* y[kSeqMaxOut];
+    void* d[kSeqMaxOut];
+    int m;
+    size_t n, head, packets;
+    SeqProgram prog;
+};
+
+template <class S>
+__global__ void __launch_bounds__(kBlock) seq_forward_kernel(const SeqForwardArgs a)
+{
+    using E = typename S::elem;
+    constexpr int V = S::kVec;
+    const size_t byte_off = a.head * sizeof(E);
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    for (size_t pk = size_t(blockIdx.x) * kBlock + threadIdx.x; pk < a.packets; pk += size_t(gridDim.x) * kBlock) {
+        uint4 raw = load_packet(reinterpret_cast<const uint4*>(static_cast<const char*>(a.x) + byte_off) + pk);
+        float xv[V], yv[kSeqMaxOut][V], yt[kSeqMaxOut][V];
+        S::unpack(raw, xv);
+        seq_run<V>(a.prog, xv, yv, yt);
+        for (int k = 0; k < a.m; ++k) {
+            *(reinterpret_cast<uint4*>(static_cast<char*>(a.y[k]) + byte_off) + pk) = S::pack(yv[k]);
+            __stcs(reinterpret_cast<uint4*>(static_cast<char*>(a.d[k]) + byte_off) + pk, S::pack(yt[k]));
+        }
+    }
+    if (blockIdx.x == 0) {
+        const size_t tail_begin = a.head + a.packets * V;
+        const size_t n_edge = a.head + (a.n - tail_begin);
+        for (size_t j = threadIdx.x; j < n_edge; j += kBlock) {
+            const size_t i = j < a.head ? j : tail_begin + (j - a.head);
+            float xv[1] = {S::load1(static_cast<const E*>(a.x) + i)};
+            float yv[kSeqMaxOut][1], yt[kSeqMaxOut][1];
+            seq_run<1>(a.prog, xv, yv, yt);
+            for (int k = 0; k < a.m; ++k) {
+                S::store1(static_cast<E*>(a.y[k]) + i, yv[k][0]);
+                S::store1(static_cast<E*>(a.d[k]) + i, yt[k][0]);
+            }
+        }
+    }
+}
+
+// Backward of a sequence with M outputs (Section II-E: the transposed Jacobian of the whole
+// sequence applied to the upstream gradients): grad_in = sum_k grad_out_k * dy_k/dx, accumulated
+// in fp32 in the order k = 0 .. m-1 with fused multiply-adds, rounded once at the store.
+struct SeqBackwardArgs {
+    const void* g[kSeqMaxOut];
+    const void* d[kSeqMaxOut];
+    void* gin;
+    int m;
+    size_t n;
+    size_t packets;    // whole 16-byte packets handled by the vector loop (0 unless every pointer is 16-byte aligned)
+};
+
+template <class S>
+__global__ void __launch_bounds__(kBlock) seq_backward_kernel(const SeqBackwardArgs a)
+{
+    using E = typename S::elem;
+    constexpr int V = S::kVec;
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    for (size_t pk = size_t(blockIdx.x) * kBlock + threadIdx.x; pk < a.packets; pk += size_t(gridDim.x) * kBlock) {
+        float acc[V], gv[V], dv[V];
+        S::unpack(load_packet(static_cast<const uint4*>(a.g[0]) + pk), gv);
+        S::unpack(load_packet(static_cast<const uint4*>(a.d[0]) + pk), dv);
+#pragma unroll
+        for (int e = 0; e < V; ++e) acc[e] = gv[e] * dv[e];
+        for (int k = 1; k < a.m; ++k) {
+            S::unpack(load_packet(static_cast<const uint4*>(a.g[k]) + pk), gv);
+            S::unpack(load_packet(static_cast<const uint4*>(a.d[k]) + pk), dv);
+#pragma unroll
+            for (int e = 0; e < V; ++e) acc[e] = fmaf(gv[e], dv[e], acc[e]);
+        }
+        *(static_cast<uint4*>(a.gin) + pk) = S::pack(acc);
+    }
+    if (blockIdx.x == 0) {
+        for (size_t i = a.packets * V + threadIdx.x; i < a.n; i += kBlock) {
+            float acc = S::load1(static_cast<const E*>(a.g[0]) + i) * S::load1(static_cast<const E*>(a.d[0]) + i);
+            for (int k = 1; k < a.m; ++k)
+                acc = fmaf(S::load1(static_cast<const E*>(a.g[k]) + i), S::load1(static_cast<const E*>(a.d[k]) + i), acc);
+            S::store1(static_cast<E*>(a.gin) + i, acc);
+        }
+    }
+}
+
+// ---------------------------------------------------------------- one operator at a time
+//
+// The same primitives as separate kernels, the way a framework runs them when every operator
+// is its own node (Section II-C approach 1): forward writes the operator's output tensor,
+// backward applies the operator's own rule to the upstream gradient and whatever the rule
+// needs (an operand or the output), which therefore has to be kept alive until then.
+struct EwArgs {
+    const void* in[3];
+    void* out[2];
+    int op;
+    int backward;
+    float c;
+    size_t n;
+    size_t packets;    // as in SeqBackwardArgs
+};
+
+__device__ __forceinline__ void ew_apply(int op, int backward, float c, float i0, float i1, float i2, float& o0, float& o1)
+{
+    const Dual<Fast> a{i0, 0.0f};
+    o1 = 0.0f;
+    if (!backward) {
+        switch (op) {
+        case kSeqAdd: o0 = i0 + i1; break;
+        case kSeqMul: o0 = i0 * i1; break;
+        case kSeqScale: o0 = c * i0; break;
+        case kSeqAddConst: o0 = c + i0; break;
+        case kSeqExp: o0 = dual_exp(a).v; break;
+        case kSeqLog1p: o0 = dual_log1p(a).v; break;
+        case kSeqTanh: o0 = dual_tanh(a).v; break;
+        case kSeqErf: o0 = dual_erf(a).v; break;
+        case kSeqSoftplus: o0 = dual_softplus(a).v; break;
+        case kSeqSigmoid: o0 = dual_sigmoid(a).v; break;
+        case kSeqHalfOnePlusTanh: o0 = dual_half_one_plus_tanh(a).v; break;
+        case kSeqHalfOnePlusErf: o0 = dual_half_one_plus_erf(a).v; break;
+        default: o0 = i0; break;
+        }
+    } else {
+        // i0 = upstream gradient; i1, i2 = what the rule kept
+        const float g = i0;
+        switch (op) {
+        case kSeqMul: o0 = g * i2; o1 = g * i1; break;                        // kept: both operands
+        case kSeqScale: o0 = c * g; break;
+        case kSeqExp: o0 = g * i1; break;                                     // kept: the output
+        case kSeqLog1p: o0 = g * hw::rcp_approx(1.0f + i1); break;            // kept: the input
+        case kSeqTanh: o0 = g * fmaf(-i1, i1, 1.0f); break;                   // kept: the output
+        case kSeqErf: o0 = g * (1.12837923f * hw::ex2_approx(-1.44269502f * (i1 * i1))); break;      // input
+        case kSeqSoftplus: o0 = g * dual_sigmoid(Dual<Fast>{i1, 0.0f}).v; break;                     // input
+        case kSeqSigmoid: o0 = g * (i1 * (1.0f - i1)); break;                 // kept: the output
+        case kSeqHalfOnePlusTanh: o0 = g * ((i1 + i1) * (1.0f - i1)); break;  // kept: the output
+        case kSeqHalfOnePlusErf: o0 = g * (0.564189613f * hw::ex2_approx(-1.44269502f * (i1 * i1))); break;   // input
+        default: o0 = g; break;
+        }
+    }
+}
+
+template <class S>
+__global__ void __launch_bounds__(kBlock) ew_kernel(const EwArgs a)
+{
+    using E = typename S::elem;
+    constexpr int V = S::kVec;
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    for (size_t pk = size_t(blockIdx.x) * kBlock + threadIdx.x; pk < a.packets; pk += size_t(gridDim.x) * kBlock) {
+        float i0[V], i1[V], i2[V], o0[V], o1[V];
+        S::unpack(load_packet(static_cast<const uint4*>(a.in[0]) + pk), i0);
+        if (a.in[1]) S::unpack(load_packet(static_cast<const uint4*>(a.in[1]) + pk), i1);
+        if (a.in[2]) S::unpack(load_packet(static_cast<const uint4*>(a.in[2]) + pk), i2);
+#pragma unroll
+        for (int e = 0; e < V; ++e) ew_apply(a.op, a.backward, a.c, i0[e], a.in[1] ? i1[e] : 0.0f, a.in[2] ? i2[e] : 0.0f, o0[e], o1[e]);
+        *(static_cast<uint4*>(a.out[0]) + pk) = S::pack(o0);
+        if (a.out[1]) *(static_cast<uint4*>(a.out[1]) + pk) = S::pack(o1);
+    }
+    if (blockIdx.x == 0) {
+        for (size_t i = a.packets * V + threadIdx.x; i < a.n; i += kBlock) {
+            float i0 = S::load1(static_cast<const E*>(a.in[0]) + i);
+            float i1 = a.in[1] ? S::load1(static_cast<const E*>(a.in[1]) + i) : 0.0f;
+            float i2 = a.in[2] ? S::load1(static_cast<const E*>(a.in[2]) + i) : 0.0f;
+            float o0, o1;
+            ew_apply(a.op, a.backward, a.c, i0, i1, i2, o0, o1);
+            S::store1(static_cast<E*>(a.out[0]) + i, o0);
+            if (a.out[1]) S::store1(static_cast<E*>(a.out[1]) + i, o1);
+        }
+    }
+}
+
+}  // namespace nfad

@@ -5,6 +5,7 @@
     python -m paper_2209_10778_b200.sweep --config resnet50   # Mish / Swish on the five ResNet-50 stage shapes
     python -m paper_2209_10778_b200.sweep --config stack      # 12 stacked GELU layers under three layouts
     python -m paper_2209_10778_b200.sweep --config probe      # plain 1:1 / 1:2 / 2:1 traffic through the same engine
+    python -m paper_2209_10778_b200.sweep --config opbyop     # nested vs operator-by-operator back-propagation, measured
 
 Each case launches one kernel `reps` times back to back between two CUDA events
 on the launching stream, after 3 warm-up launches; buffers are rotated so that
@@ -130,6 +131,60 @@ def run_probe(n_words: int, reps: int = 20, dev="cuda"):
     return out
 
 
+def run_opbyop(n: int, dtype: str, kinds, reps: int = 5, dev="cuda"):
+    """Forward + backward of each activation under four executions of the SAME function: the
+    dedicated nested kernels, the run-time FAD sequence (one generic kernel), and operator-by-
+    operator back-propagation (one kernel per primitive, every rule keeping what it needs) --
+    the layout the paper's memory comparison is made against.  Reports kept bytes and time."""
+    from . import sequence
+    out = []
+    x = W.normal(n, dtype, 0, 1.0, dev)
+    g = W.normal(n, dtype, 1, 1.0, dev)
+    es = x.element_size()
+
+    def timed(fn):
+        fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / reps
+
+    for kind in kinds:
+        prog = sequence.PROGRAMS[kind]()
+        y, d, gin = torch.empty_like(x), torch.empty_like(x), torch.empty_like(x)
+
+        def nested():
+            nfad.nfad_act_forward(kind, x, y, d)
+            nfad.nfad_act_backward(kind, g, d, gin)
+
+        def fused_seq():
+            nfad.nfad_seq_forward(prog.ops, x, [y], [d])
+            nfad.nfad_seq_backward([g], [d], gin)
+
+        ex = sequence.OpByOp(prog)
+        kept = {}
+
+        def op_by_op():
+            ex.forward(x)
+            kept["bytes"] = ex.saved_bytes()
+            ex.backward([g])
+
+        rows = [("nested (dedicated kernels)", nested, n * es), ("nested (run-time sequence)", fused_seq, n * es),
+                ("operator by operator", op_by_op, None)]
+        for name, fn, saved in rows:
+            ms = timed(fn)
+            out.append({"config": "opbyop", "kind": kind, "dtype": dtype, "n": n, "execution": name, "ms_fwd_bwd": ms,
+                        "kept_bytes": saved if saved is not None else kept["bytes"],
+                        "kept_tensors": (saved if saved is not None else kept["bytes"]) / (n * es),
+                        "launches": 2 if saved is not None else None})
+            torch.cuda.empty_cache()
+    return out
+
+
 def run_stack(layers: int, n: int, dtype: str, kind: str, dev="cuda", reps: int = 3):
     """L stacked activations: forward through all layers, then backward in reverse, under the three
     layouts; reports the bytes kept alive between the passes and the total device time."""
@@ -193,7 +248,7 @@ def run_stack(layers: int, n: int, dtype: str, kind: str, dev="cuda", reps: int 
 
 def main(argv=None):
     ap = argparse.ArgumentParser()
-    ap.add_argument("--config", default=None, choices=[None, "sizes", "resnet50", "stack", "bert", "probe"])
+    ap.add_argument("--config", default=None, choices=[None, "sizes", "resnet50", "stack", "bert", "probe", "opbyop"])
     ap.add_argument("--n", type=int, default=100663296)
     ap.add_argument("--kinds", default="gelu_erf,gelu_tanh,swish,mish")
     ap.add_argument("--dtypes", default="bf16")
@@ -233,6 +288,10 @@ def main(argv=None):
     elif args.config == "probe":
         for r in run_probe(args.n // 2, args.reps):          # n bf16-sized elements -> n/2 words
             print(json.dumps(r), flush=True)
+    elif args.config == "opbyop":
+        for dtype in dtypes:
+            for r in run_opbyop(args.n, dtype, kinds):
+                print(json.dumps(r), flush=True)
     elif args.config == "stack":
         w = W.WORKLOADS["gelu_stack_12"]
         for r in run_stack(w.layers, w.numel(0), w.dtype, w.kinds[0]):

@@ -1,0 +1,188 @@
+"""GPU tests of run-time FAD sequences: the fused executor and the operator-by-operator
+executor against the fp64 sequence oracle, the M-result backward, the autograd wrappers.
+
+Tolerance of this executor (plain fp32 primitives for every storage type, no hardening):
+  fp32     |got - o| <= 2e-5 * max(|o|, S) with S the size of the largest intermediate sum
+           feeding the result (taken as 1 + |x| here), i.e. a few fp32 ulp of the terms;
+  16-bit   within 1 ulp of the rounded oracle value, or within the fp32 tolerance above.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import ulp
+from paper_2209_10778_b200 import autograd as nfad_autograd
+from paper_2209_10778_b200 import binding as nfad
+from paper_2209_10778_b200 import sequence
+from paper_2209_10778_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+def _two_result_program():
+    # results: sigmoid(x) * tanh(x)   and   exp(-x^2/2-ish) + x : merges of same-source branches, M = 2
+    p = sequence.FadProgram()
+    x = p.x()
+    a = p.mul(p.unary("sigmoid", x), p.unary("tanh", x))
+    b = p.add(p.unary("exp", p.scale(-0.5, p.mul(x, x))), x)
+    p.output(a)
+    p.output(b)
+    return p
+
+
+PROGRAMS = {
+    "swish": sequence.swish_program, "mish": sequence.mish_program, "gelu_tanh": sequence.gelu_tanh_program,
+    "gelu_erf": sequence.gelu_erf_program, "gelu_tanh_literal": sequence.gelu_tanh_literal_program,
+    "two_results": _two_result_program,
+    "log1p_softplus_erf": lambda: (lambda p: (p.output(p.add(p.unary("log1p", p.unary("softplus", p.x())), p.unary("erf", p.x()))), p)[1])(sequence.FadProgram()),
+}
+
+
+def _close(dtype, got_t, want64, x64):
+    got_raw = W.raw_numpy(got_t)
+    got = oracle.widen(dtype, got_raw)
+    tol32 = 2e-5 * np.maximum(np.abs(want64), 1.0 + np.abs(x64))
+    ok = np.abs(got - want64) <= tol32
+    if dtype != "f32":
+        ok |= ulp.ulp_distance16(got_raw, oracle.round_to(dtype, want64)) <= 1
+    return ok
+
+
+@pytest.mark.parametrize("name", list(PROGRAMS))
+@pytest.mark.parametrize("dtype", ["f32", "bf16", "f16"])
+def test_fused_executor_against_the_sequence_oracle(name, dtype):
+    prog = PROGRAMS[name]()
+    n = 70001
+    x = (W.normal(n, "f32", 5, 2.0, DEV).clamp_(-7, 7)).to(W.TORCH_DTYPES[dtype])
+    ys, ds = sequence.run_fused(prog, x)
+    torch.cuda.synchronize()
+    x64 = oracle.widen(dtype, W.raw_numpy(x))
+    y, d = oracle.seq_forward(prog.ops, x64, prog.n_out)
+    for k in range(prog.n_out):
+        assert _close(dtype, ys[k], y[k], x64).all(), (name, dtype, "value", k)
+        assert _close(dtype, ds[k], d[k], x64).all(), (name, dtype, "derivative", k)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16", "f16"])
+def test_fused_executor_edges_and_unaligned(dtype):
+    prog = sequence.swish_program()
+    td = W.TORCH_DTYPES[dtype]
+    for n in (1, 7, 8, 9, 255, 257, 4099):
+        buf = W.normal(n + 16, dtype, n, 1.0, DEV)
+        for off in (0, 1, 3):
+            x = buf[off:off + n]
+            yb = torch.full((n + 16,), 7.0, dtype=td, device=DEV)
+            db = torch.full((n + 16,), 7.0, dtype=td, device=DEV)
+            nfad.nfad_seq_forward(prog.ops, x, [yb[off:off + n]], [db[off + 1:off + 1 + n]] if off == 3 else [db[off:off + n]])
+            torch.cuda.synchronize()
+            x64 = oracle.widen(dtype, W.raw_numpy(x))
+            y, d = oracle.seq_forward(prog.ops, x64, 1)
+            assert _close(dtype, yb[off:off + n], y[0], x64).all()
+            assert (yb[:off] == 7.0).all() and (yb[off + n:] == 7.0).all()
+            dsl = db[off + 1:off + 1 + n] if off == 3 else db[off:off + n]
+            assert _close(dtype, dsl, d[0], x64).all()
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16", "f16"])
+def test_backward_of_a_two_result_sequence(dtype):
+    prog = _two_result_program()
+    n = 50003
+    x = W.normal(n, dtype, 7, 1.5, DEV)
+    gs = [W.normal(n, dtype, 8 + k, 1.0, DEV) for k in range(2)]
+    ys, ds = sequence.run_fused(prog, x)
+    gin = sequence.backward_fused(gs, ds)
+    torch.cuda.synchronize()
+    g64 = np.stack([oracle.widen(dtype, W.raw_numpy(g)) for g in gs])
+    d64 = np.stack([oracle.widen(dtype, W.raw_numpy(d)) for d in ds])       # the GPU's own saved derivatives
+    s, sa = oracle.seq_backward(g64, d64)
+    got_raw = W.raw_numpy(gin)
+    got = oracle.widen(dtype, got_raw)
+    # fp32 accumulation of exact products: one fp32 rounding per term of size <= sa, then the store's rounding
+    tol = 2.0 ** -23 * sa
+    ok = np.abs(got - s) <= tol
+    if dtype != "f32":
+        ok |= ulp.ulp_distance16(got_raw, oracle.round_to(dtype, s)) <= 1
+    assert ok.all()
+    # m == 1 is the plain backward, bit for bit
+    one = sequence.backward_fused(gs[:1], ds[:1])
+    ref = torch.empty_like(one)
+    nfad.nfad_act_backward("swish", gs[0], ds[0], ref)
+    torch.cuda.synchronize()
+    assert np.array_equal(W.raw_numpy(one), W.raw_numpy(ref))
+
+
+@pytest.mark.parametrize("name", ["swish", "gelu_tanh", "mish", "two_results"])
+def test_operator_by_operator_executor(name):
+    dtype = "f32"
+    prog = PROGRAMS[name]()
+    n = 40009
+    x = W.normal(n, "f32", 9, 1.5, DEV).clamp_(-6, 6)
+    ex = sequence.OpByOp(prog)
+    outs = ex.forward(x)
+    kept = ex.saved_bytes()
+    gs = [W.normal(n, dtype, 20 + k, 1.0, DEV) for k in range(prog.n_out)]
+    gin = ex.backward(gs)
+    torch.cuda.synchronize()
+    x64 = oracle.widen(dtype, W.raw_numpy(x))
+    y, d = oracle.seq_forward(prog.ops, x64, prog.n_out)
+    for k in range(prog.n_out):
+        assert _close(dtype, outs[k], y[k], x64).all()
+    g64 = np.stack([oracle.widen(dtype, W.raw_numpy(g)) for g in gs])
+    s, sa = oracle.seq_backward(g64, d)
+    got = oracle.widen(dtype, W.raw_numpy(gin))
+    assert (np.abs(got - s) <= 4e-5 * np.maximum(sa, np.abs(g64).sum(0) * (1 + np.abs(x64)))).all()
+    # what operator-by-operator back-propagation keeps: Swish keeps x and sigmoid(x) (the paper's v1, v2)
+    if name == "swish":
+        assert kept == 2 * n * 4
+    assert kept >= 2 * n * 4
+
+
+def test_autograd_wrappers():
+    n = 7 * 2859
+    for kind, fn in (("gelu_erf", lambda t: nfad_autograd.gelu(t)), ("gelu_tanh", lambda t: nfad_autograd.gelu(t, "tanh")),
+                     ("swish", nfad_autograd.silu), ("mish", nfad_autograd.mish)):
+        x = W.normal(n, "bf16", 3, 1.5, DEV).view(7, -1).requires_grad_(True)
+        g = W.normal(n, "bf16", 4, 1.0, DEV).view(7, -1)
+        y = fn(x)
+        y.backward(g)
+        y0, d0, gin0 = torch.empty(n, dtype=x.dtype, device=DEV), torch.empty(n, dtype=x.dtype, device=DEV), torch.empty(n, dtype=x.dtype, device=DEV)
+        nfad.nfad_act_forward(kind, x.detach().view(-1), y0, d0)
+        nfad.nfad_act_backward(kind, g.view(-1), d0, gin0)
+        torch.cuda.synchronize()
+        assert torch.equal(y.detach().view(-1), y0) and torch.equal(x.grad.view(-1), gin0)
+        # the conventional wrapper gives the same value and a gradient within one bf16 ulp-ish of it
+        x2 = x.detach().clone().requires_grad_(True)
+        y2 = nfad_autograd.ConventionalActivation.apply(x2, kind)
+        y2.backward(g)
+        torch.cuda.synchronize()
+        assert torch.equal(y2.detach(), y.detach())
+        assert torch.allclose(x2.grad.float(), x.grad.float(), rtol=2e-2, atol=1e-3)
+    # a two-result sequence through autograd
+    prog = _two_result_program()
+    x = W.normal(n, "f32", 5, 1.0, DEV).requires_grad_(True)
+    a, b = nfad_autograd.FadSequence.apply(x, prog)
+    (a.sum() * 2.0 + b.sum()).backward()
+    torch.cuda.synchronize()
+    x64 = x.detach().double().cpu().numpy()
+    y, d = oracle.seq_forward(prog.ops, x64, 2)
+    want = 2.0 * d[0] + d[1]
+    assert np.allclose(x.grad.double().cpu().numpy(), want, rtol=2e-5, atol=2e-5)
+
+
+def test_malformed_programs_are_refused():
+    x = torch.zeros(64, device=DEV)
+    y, d = torch.zeros(64, device=DEV), torch.zeros(64, device=DEV)
+    bad = [
+        [("exp", 3, 3, 1, 0.0), ("out", 1, 1, 0, 0.0)],          # reads a register nobody wrote
+        [("exp", 0, 0, 1, 0.0), ("out", 1, 1, 1, 0.0)],          # result slot out of range
+        [("exp", 0, 0, 0, 0.0), ("out", 0, 0, 0, 0.0)],          # writes the source register
+        [("exp", 0, 0, 1, 0.0)],                                 # produces no result
+        [(99, 0, 0, 1, 0.0), ("out", 1, 1, 0, 0.0)],             # unknown opcode
+    ]
+    for prog in bad:
+        with pytest.raises(nfad.NfadError) as e:
+            nfad.nfad_seq_forward(prog, x, [y], [d])
+        assert e.value.status == 10
+    torch.cuda.synchronize()
