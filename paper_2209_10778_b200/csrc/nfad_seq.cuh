@@ -52,24 +52,36 @@ __device__ __forceinline__ Dual<Fast> seq_apply(const SeqOp& o, const Dual<Fast>
     }
 }
 
+// Interprets the program for V elements, kSeqGroup at a time: the register file is indexed at
+// run time and so lives in local memory, and kSeqRegs x 2 x kSeqGroup floats per thread is what
+// has to stay inside L1 for every resident thread.
+#ifndef NFAD_SEQ_GROUP
+#define NFAD_SEQ_GROUP 2
+#endif
+constexpr int kSeqGroup = NFAD_SEQ_GROUP;
+
 template <int V>
 __device__ __forceinline__ void seq_run(const SeqProgram& prog, const float (&x)[V], float (&yv)[kSeqMaxOut][V],
                                         float (&yt)[kSeqMaxOut][V])
 {
-    float rv[kSeqRegs][V], rt[kSeqRegs][V];
+    constexpr int G = V < kSeqGroup ? V : kSeqGroup;
 #pragma unroll
-    for (int e = 0; e < V; ++e) { rv[0][e] = x[e]; rt[0][e] = 1.0f; }
-    for (int i = 0; i < prog.n_ops; ++i) {
-        const SeqOp o = prog.ops[i];
-        if (o.op == kSeqOut) {
+    for (int e0 = 0; e0 < V; e0 += G) {
+        float rv[kSeqRegs][G], rt[kSeqRegs][G];
 #pragma unroll
-            for (int e = 0; e < V; ++e) { yv[o.dst][e] = rv[o.a][e]; yt[o.dst][e] = rt[o.a][e]; }
-        } else {
+        for (int e = 0; e < G; ++e) { rv[0][e] = x[e0 + e]; rt[0][e] = 1.0f; }
+        for (int i = 0; i < prog.n_ops; ++i) {
+            const SeqOp o = prog.ops[i];
+            if (o.op == kSeqOut) {
 #pragma unroll
-            for (int e = 0; e < V; ++e) {
-                Dual<Fast> r = seq_apply(o, Dual<Fast>{rv[o.a][e], rt[o.a][e]}, Dual<Fast>{rv[o.b][e], rt[o.b][e]});
-                rv[o.dst][e] = r.v;
-                rt[o.dst][e] = r.t;
+                for (int e = 0; e < G; ++e) { yv[o.dst][e0 + e] = rv[o.a][e]; yt[o.dst][e0 + e] = rt[o.a][e]; }
+            } else {
+#pragma unroll
+                for (int e = 0; e < G; ++e) {
+                    Dual<Fast> r = seq_apply(o, Dual<Fast>{rv[o.a][e], rt[o.a][e]}, Dual<Fast>{rv[o.b][e], rt[o.b][e]});
+                    rv[o.dst][e] = r.v;
+                    rt[o.dst][e] = r.t;
+                }
             }
         }
     }
