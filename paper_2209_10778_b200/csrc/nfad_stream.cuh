@@ -5,10 +5,10 @@
 // enough of them in flight to cover HBM latency, and (2) spend as few issue
 // slots per element as possible between the load and the store.
 //
-// Work decomposition: a tile is kBlock * kUnroll consecutive packets; thread t
+// Work decomposition: a tile is kBlock * U consecutive packets (U = 4, or the op's choice); thread t
 // of a CTA owns packets t, t + kBlock, ... of the tile, so every warp-level
 // access is one contiguous 512-byte run.  One CTA per tile; each thread issues
-// all kUnroll * NIN loads of its tile before the first use.  Elements before the first and after the
+// all U * NIN loads of its tile before the first use.  Elements before the first and after the
 // last whole packet (unaligned base, ragged tail) are handled one by one by the
 // first warps of CTA 0 with the very same per-element code, so the vector and
 // scalar paths agree bit for bit.
@@ -25,7 +25,7 @@ constexpr int kBlock = 256;
 #ifndef NFAD_UNROLL
 #define NFAD_UNROLL 4
 #endif
-constexpr int kUnroll = NFAD_UNROLL;
+constexpr int kDefaultUnroll = NFAD_UNROLL;
 // Resident CTAs per SM the compiler must leave room for (a register cap).  The 16-bit kernels
 // are issue-bound with short dependency chains through MUFU: 5 CTAs (40 warps, <= 48 registers)
 // measured 3-5 % faster than the 4 the compiler picks by itself (7 or more spill and lose 30 %); the fp32 kernels need their
@@ -140,6 +140,7 @@ template <int NIN, int NOUT> struct StreamArgs {
 //   static constexpr int kIn, kOut;  static constexpr bool keep(int out_slot);
 //   static __device__ void apply(const float (&in)[kIn], float (&out)[kOut]);
 //   static constexpr int kMinBlocks: resident CTAs per SM to leave room for (0: the storage type's default);
+//   static constexpr int kUnroll: packets per thread and tile (0: the default, 4);
 //   static constexpr bool kPacketFixup; if set, fixup(vin, vout) may patch a whole packet's
 //   results after apply (a rare case kept off the per-element path) and apply_checked is the
 //   one-element form that includes the patch.
@@ -185,10 +186,14 @@ __device__ __forceinline__ void packet_compute_store(const StreamArgs<Op::kIn, O
     }
 }
 
+// Packets per thread and tile: the op's own choice if it states one, else the default.
+template <class Op> struct UnrollOf { static constexpr int value = Op::kUnroll ? Op::kUnroll : kDefaultUnroll; };
+
 template <class S, class Op>
 __global__ void __launch_bounds__(kBlock, (Op::kMinBlocks ? Op::kMinBlocks : S::kMinBlocks)) stream_kernel(const StreamArgs<Op::kIn, Op::kOut> a)
 {
     constexpr int V = S::kVec;
+    constexpr int kUnroll = UnrollOf<Op>::value;
     const size_t byte_off = a.head * sizeof(typename S::elem);
     const size_t tile_packets = size_t(kBlock) * kUnroll;
     const size_t n_tiles = (a.packets + tile_packets - 1) / tile_packets;
@@ -313,7 +318,7 @@ cudaError_t launch_stream(const void* const* in, void* const* out, size_t n, cud
     if (head > n) head = n;
     a.head = head;
     a.packets = (n - head) / S::kVec;
-    const size_t tile_packets = size_t(kBlock) * kUnroll;
+    const size_t tile_packets = size_t(kBlock) * UnrollOf<Op>::value;
     size_t tiles = (a.packets + tile_packets - 1) / tile_packets;
     if (tiles == 0) tiles = 1;                                  // edges only
     // One tile per CTA, handed out in address order by the hardware as CTAs retire: measured
