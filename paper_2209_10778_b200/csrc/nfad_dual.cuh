@@ -156,17 +156,31 @@ NFAD_DEV Gate<Fast> logistic_fast(float w, float minus_log2e_scale, float slope_
 
 // Full: |w| = -(ah + al).  For w < 0 the common factor 2^n of e is left out of
 // value and slope (they carry it as `sc`); for w >= 0 the value is the pair (1, -small).
+// The exponential comes as 2^n (1 + g) and is applied as m (1 + g) = fmaf(m, g, m), so 1 + g is
+// never rounded; 1/(1+e) is a Newton-refined reciprocal of the exactly known 1 + e.  Every fp32
+// input was run against the fp64 oracle with this arithmetic (see tests/certify_fp32_exhaustive.py).
+// kFineSlope spends six more instructions on the slope (two-float 1/(1+e), its square formed
+// exactly): needed where the slope is multiplied by a large chain-rule factor, as in GELU-tanh.
+template <bool kFineSlope>
 NFAD_DEV Gate<Full> logistic_full(float ah, float al, bool neg)
 {
-    ExpParts E = exp_parts_full(ah, al);
+    ExpG E = exp_g_full(ah, al);
     float sc = pow2_clamped(E.n);
-    float eh = E.p.h * sc;
-    float dh = 1.0f + eh;
-    float dl = fmaf(E.p.l, sc, eh - (dh - 1.0f));   // 1 + e = dh + dl
-    F2 big = f2_rcp(F2{dh, dl});               // 1/(1+e)
-    F2 pr = f2_mul(E.p, big);                  // small / 2^n
-    float dd = fmaf(pr.h, big.h, fmaf(pr.l, big.h, pr.h * big.l));   // big small / 2^n, one rounding
-    F2 v = neg ? pr : F2{1.0f, -(f2_value(pr) * sc)};
+    float e = fmaf(sc, E.g, sc);
+    float dh = 1.0f + e;
+    float dl = e - (dh - 1.0f);                // 1 + e = dh + dl
+    F2 big2 = f2_rcp(F2{dh, dl});              // 1/(1+e); the low part is dead code unless kFineSlope
+    float big = big2.h;
+    float pr = fmaf(big, E.g, big);            // small / 2^n
+    float dd;                                  // big small / 2^n
+    if (kFineSlope) {
+        F2 bb = two_prod(big, big);
+        bb.l = fmaf(big + big, big2.l, bb.l);  // 1/(1+e)^2
+        dd = fmaf(bb.h, E.g, bb.h) + bb.l;
+    } else {
+        dd = pr * big;
+    }
+    F2 v = neg ? F2{pr, 0.0f} : F2{1.0f, -(pr * sc)};
     float d = neg ? dd : dd * sc;
     return {v, d, neg ? sc : 1.0f, neg ? E.n : 0};
 }
@@ -181,7 +195,7 @@ template <class In> NFAD_DEV Gate<Full> dual_sigmoid_full(const In& a)
 {
     F2 v = in_v2(a);
     bool neg = v.h < 0.0f;
-    Gate<Full> g = logistic_full(-fabsf(v.h), neg ? v.l : -v.l, neg);
+    Gate<Full> g = logistic_full<false>(-fabsf(v.h), neg ? v.l : -v.l, neg);
     return {g.v, chain(g.t, a), g.sc, g.n};
 }
 NFAD_DEV Gate<Fast> dual_sigmoid(Fast, const Seed& a) { return dual_sigmoid_fast(a); }
@@ -200,7 +214,7 @@ NFAD_DEV Gate<Full> dual_half_one_plus_tanh(const Dual<Full>& u)
 {
     bool neg = u.v.h < 0.0f;
     float two_ul = u.v.l + u.v.l;
-    Gate<Full> g = logistic_full(-2.0f * fabsf(u.v.h), neg ? two_ul : -two_ul, neg);
+    Gate<Full> g = logistic_full<true>(-2.0f * fabsf(u.v.h), neg ? two_ul : -two_ul, neg);
     return {g.v, chain(g.t + g.t, u), g.sc, g.n};
 }
 

@@ -148,6 +148,31 @@ NFAD_DEV ExpParts exp_parts_full(float ah, float al)
     return {{ph, pl}, ni};
 }
 
+// Leaner variant: e^(ah+al) = 2^n (1 + g) with g one float (|g| < 0.42), good to ~0.4 units of
+// 2^-24 relative to the result.  Callers multiply by (1 + g) with one fused multiply-add,
+// m (1 + g) = fmaf(m, g, m), so that 1 + g itself is never rounded.
+struct ExpG { float g; int n; };
+
+NFAD_DEV ExpG exp_g_full(float ah, float al)
+{
+    const float kLog2e = 1.44269502f;
+    const float kMagic = 12582912.0f;
+    const float kLn2Hi = 0.693147182f;
+    const float kLn2Lo = -1.90465421e-09f;
+    float t = fmaf(ah, kLog2e, kMagic);
+    float n = t - kMagic;
+    int ni = hw::float_as_int(t) - 0x4B400000;
+    float rh = fmaf(n, -kLn2Hi, ah);           // exact
+    float r = rh + fmaf(n, -kLn2Lo, al);
+    float q = 0.000199696486f;
+    q = fmaf(q, r, 0.00139308674f);
+    q = fmaf(q, r, 0.0083331801f);
+    q = fmaf(q, r, 0.0416665077f);
+    q = fmaf(q, r, 0.166666672f);
+    q = fmaf(q, r, 0.5f);
+    return {fmaf(r * r, q, r), ni};
+}
+
 // ---------------------------------------------------------------- exp, Fast
 
 
