@@ -19,6 +19,9 @@
 // free of cancellation:
 //     dual_half_one_plus_tanh(u) = (1 + tanh u)/2 = sigmoid(2u)
 //     dual_half_one_plus_erf(z)  = (1 + erf z)/2  = erfc(-z)/2
+// and one fusion of mul / scale / add_const over the seed alone, with its derivative
+// in closed form like any other primitive:
+//     dual_odd_cubic(c1, c3, x)  = c1 x + c3 x^3,  tangent c1 + 3 c3 x^2
 //
 // Policies.  Fast (16-bit storage): a value and a tangent are one float each.
 // Full (fp32 storage): values and the tangents of the polynomial part of a
@@ -50,6 +53,11 @@ template <> struct Gate<Full> { F2 v; float t; float sc; int n; };   // (v, t) t
 
 // A constant known to more than fp32 precision.
 struct Const2 { float h, l; };
+// The same, split so that the high part is a positive multiple of 2^-20 (and the low part
+// correspondingly larger).  For e >= 0 and s = fl(h + e) < 16 the difference s - h is then
+// exact (a multiple of s's last place that fits 24 bits), which makes the rounding error of
+// a fused multiply-add onto h recoverable with one more fused multiply-add.
+struct SplitConst { float h, l; };
 
 NFAD_DEV float dual_value(const Dual<Fast>& a) { return a.v; }
 NFAD_DEV float dual_tangent(const Dual<Fast>& a) { return a.t; }
@@ -125,6 +133,32 @@ NFAD_DEV Dual<Fast> dual_mul(const Dual<Fast>& a, const Dual<Fast>& b)
 NFAD_DEV Dual<Full> dual_mul(const Dual<Full>& a, const Dual<Full>& b)
 {
     return {f2_mul(a.v, b.v), f2_add(f2_mul(a.v, b.t), f2_mul(a.t, b.v))};
+}
+
+// ----------------------------------------------------------------- odd cubic of the seed
+//
+// p(x) = c1 x + c3 x^3 = x (c1 + c3 x^2),  p'(x) = c1 + 3 c3 x^2   (k3 = 3 c3 is passed in).
+// Full: both brackets are formed as two-floats from the exact square x^2 = s.h + s.l; the
+// high part is one fused multiply-add onto c1.h and the low part recovers its rounding error
+// (see SplitConst) plus the terms of the constants' and the square's low parts.  Needs
+// c1 + k x^2 < 15.
+NFAD_DEV F2 cubic_bracket(SplitConst c1, Const2 k, F2 s)
+{
+    float h = fmaf(k.h, s.h, c1.h);
+    float l = fmaf(k.h, s.h, c1.h - h);
+    l += fmaf(k.h, s.l, fmaf(k.l, s.h, c1.l));
+    return {h, l};
+}
+NFAD_DEV Dual<Full> dual_odd_cubic(Full, SplitConst c1, Const2 c3, Const2 k3, const Seed& a)
+{
+    F2 s = two_prod(a.x, a.x);
+    return {f2_mul(cubic_bracket(c1, c3, s), a.x), cubic_bracket(c1, k3, s)};
+}
+NFAD_DEV Dual<Fast> dual_odd_cubic(Fast, SplitConst c1, Const2 c3, Const2 k3, const Seed& a)
+{
+    float s = a.x * a.x;
+    float c = c1.h + c1.l;
+    return {a.x * fmaf(c3.h, s, c), fmaf(k3.h, s, c)};
 }
 
 // ----------------------------------------------------------------- chain rule's last factor
@@ -394,13 +428,11 @@ template <class P> NFAD_DEV Gate<P> gate(GeluErf, Seed X)
 // GELU, tanh form (Table I): h = (1 + tanh(sqrt(2/pi) (x + 0.044715 x^3)))/2
 template <class P> NFAD_DEV Gate<P> gate(GeluTanh, Seed X)
 {
-    const Const2 kA = {0.044714998453855515f, 1.5461444e-09f};   // 0.044715
-    const Const2 kC = {0.7978845834732056f, -2.2670340e-08f};    // sqrt(2/pi)
-    Dual<P> X2 = dual_mul(P{}, X, X);
-    Dual<P> B = dual_add_const(1.0f, dual_scale(kA, X2));   // 1 + a x^2
-    Dual<P> Q = dual_mul(X, B);                             // x + a x^3
-    Dual<P> U = dual_scale(kC, Q);
-    return dual_half_one_plus_tanh(U);
+    // u = c x + (c a) x^3 with c = sqrt(2/pi), a = 0.044715 (the double nearest to it)
+    const SplitConst kC = {0.7978849411010742f, -3.8029822e-07f};
+    const Const2 kCA = {0.035677406936883926f, 1.1994162e-09f};
+    const Const2 k3CA = {0.10703222453594208f, -1.2704171e-10f};
+    return dual_half_one_plus_tanh(dual_odd_cubic(P{}, kC, kCA, k3CA, X));
 }
 
 // Swish (Table I, Table II): h = sigmoid(x)
@@ -419,7 +451,7 @@ struct ActOut { float y, dydx; };
 // of the tanh form).
 template <class K> struct Saturation;
 template <> struct Saturation<GeluErf> { static constexpr float kFull = 20.0f; static constexpr bool kFastClamp = false; };
-template <> struct Saturation<GeluTanh> { static constexpr float kFull = 20.0f; static constexpr bool kFastClamp = true; };
+template <> struct Saturation<GeluTanh> { static constexpr float kFull = 11.5f; static constexpr bool kFastClamp = true; };
 template <> struct Saturation<Swish> { static constexpr float kFull = 120.0f; static constexpr bool kFastClamp = false; };
 template <> struct Saturation<Mish> { static constexpr float kFull = 120.0f; static constexpr bool kFastClamp = false; };
 
