@@ -6,8 +6,9 @@ library never does, and this package imports nothing of the CUDA library.
 
 The arithmetic lives in ``nfad_oracle.c`` (plain C, fp64, one expression per
 quantity: Table I for the activations, Table II / Eq. 3 for the derivatives,
-Eq. 4 for the backward product).  This module compiles that file with gcc on
-first use and marshals numpy arrays into it.  Stored tensors cross the boundary
+Eq. 4 for the backward product), ``nfad_seq_oracle.c`` (run-time FAD sequences)
+and ``nfad_bias_oracle.c`` (the pass with its producer's bias-add and the bias
+gradient).  This module compiles those files with gcc on first use and marshals numpy arrays into it.  Stored tensors cross the boundary
 as raw bit patterns: ``float32`` arrays for fp32, ``uint16`` arrays for bf16 and
 fp16.
 """
@@ -26,6 +27,7 @@ DTYPES = {"f32": 0, "bf16": 1, "f16": 2}
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "nfad_oracle.c")
 _SRC_SEQ = os.path.join(_HERE, "nfad_seq_oracle.c")
+_SRC_BIAS = os.path.join(_HERE, "nfad_bias_oracle.c")
 _LIB = os.path.join(_HERE, "libnfad_oracle.so")
 _lock = threading.Lock()
 _lib = None
@@ -34,10 +36,10 @@ _lib = None
 def build(force: bool = False) -> str:
     """Compile the oracle with gcc (IEEE semantics: no fast-math, no contraction)."""
     with _lock:
-        stale = (not os.path.exists(_LIB)) or os.path.getmtime(_LIB) < max(os.path.getmtime(_SRC), os.path.getmtime(_SRC_SEQ))
+        stale = (not os.path.exists(_LIB)) or os.path.getmtime(_LIB) < max(os.path.getmtime(f) for f in (_SRC, _SRC_SEQ, _SRC_BIAS))
         if force or stale:
             cmd = ["gcc", "-O2", "-std=c11", "-fPIC", "-shared", "-fopenmp",
-                   "-ffp-contract=off", "-fno-fast-math", "-o", _LIB, _SRC, _SRC_SEQ, "-lm"]
+                   "-ffp-contract=off", "-fno-fast-math", "-o", _LIB, _SRC, _SRC_SEQ, _SRC_BIAS, "-lm"]
             subprocess.run(cmd, check=True, capture_output=True)
     return _LIB
 
@@ -69,6 +71,10 @@ def _load():
         lib.nfad_seq_oracle_forward.restype = ci
         lib.nfad_seq_oracle_backward.argtypes = [vp, vp, sz, ci, vp, vp]
         lib.nfad_seq_oracle_backward.restype = ci
+        lib.nfad_bias_oracle_forward.argtypes = [ci, ci, vp, vp, sz, sz, vp, vp, vp, vp]
+        lib.nfad_bias_oracle_forward.restype = ci
+        lib.nfad_bias_oracle_backward.argtypes = [ci, vp, vp, sz, sz, vp, vp, vp]
+        lib.nfad_bias_oracle_backward.restype = ci
         _lib = lib
     return _lib
 
@@ -202,3 +208,32 @@ def seq_backward(g: np.ndarray, d: np.ndarray):
     out_abs = np.empty(n, np.float64)
     _ok(_load().nfad_seq_oracle_backward(_ptr(g), _ptr(d), n, m, _ptr(out), _ptr(out_abs)), "seq_backward")
     return out, out_abs
+
+
+def bias_forward(kind, dtype, x: np.ndarray, bias: np.ndarray, rows: int, cols: int, want_cond: bool = False):
+    """Unrounded f(z), f'(z) in fp64 at z = fl32(x[r, c] + bias[c]) for a row-major [rows, cols] stored tensor x
+    and a stored bias of cols elements.  Returns (f, f', z) or (f, f', z, |h| + |z h'|), flat."""
+    x = _check_storage(x, dtype)
+    bias = _check_storage(bias, dtype)
+    if x.size != rows * cols or bias.size != cols:
+        raise ValueError("size mismatch")
+    f, fp, z = (np.empty(x.size, np.float64) for _ in range(3))
+    cond = np.empty(x.size, np.float64) if want_cond else None
+    _ok(_load().nfad_bias_oracle_forward(_code(KINDS, kind), _code(DTYPES, dtype), _ptr(x), _ptr(bias), rows, cols,
+                                         _ptr(f), _ptr(fp), _ptr(cond) if want_cond else None, _ptr(z)), "bias_forward")
+    return (f, fp, z, cond) if want_cond else (f, fp, z)
+
+
+def bias_backward(dtype, grad_out: np.ndarray, fprime_saved: np.ndarray, rows: int, cols: int):
+    """(grad_in stored, grad_bias fp64, sum of |grad_in| per column fp64): grad_in = RN(grad_out * f'_saved) and
+    grad_bias[c] = sum over rows of the rounded grad_in[r, c] (Eq. 4 for x; dz/db = 1 for the bias)."""
+    g = _check_storage(grad_out, dtype)
+    d = _check_storage(fprime_saved, dtype)
+    if g.size != rows * cols or d.size != rows * cols:
+        raise ValueError("size mismatch")
+    gin = np.empty(g.size, _storage_np(dtype))
+    gb = np.empty(cols, np.float64)
+    gb_abs = np.empty(cols, np.float64)
+    _ok(_load().nfad_bias_oracle_backward(_code(DTYPES, dtype), _ptr(g), _ptr(d), rows, cols, _ptr(gin), _ptr(gb),
+                                          _ptr(gb_abs)), "bias_backward")
+    return gin, gb, gb_abs
