@@ -244,6 +244,49 @@ NFAD_API int nfad_ew_op(int op, int backward, float c, int dtype, const void* in
                         void* out0, void* out1, size_t n, nfad_stream_t stream);
 
 /*
+ * The pass fused with its producer's bias.
+ *
+ * A linear layer hands over x[rows, cols] (row-major, contiguous) and bias[cols]; the
+ * activation sees z = x + bias.  From x's side the addition is a binary operation with
+ * one constant input, which the method treats as unary (Section III-A), and dz/dx = 1:
+ * the forward pass still emits y = f(z) and the one saved tensor f'(z), and the backward
+ * pass is still the multiplication of Eq. 4.  From the bias's side dz/dbias = 1 on every
+ * row, so its gradient is the column sum of that same product.  The paper only notes
+ * that frameworks fuse such element-wise chains by hand (Section III); these two entry
+ * points are that fusion for this library, and save one write and one read of the
+ * pre-activation tensor forward and one read of grad_in backward.
+ *
+ * Forward:  z = x[r, c] + bias[c], formed by ONE fp32 addition (for every storage type);
+ *           y[r, c] = f(z), dfdx[r, c] = f'(z), arithmetic and rounding as nfad_act_forward.
+ *   x [in] rows*cols elements; bias [in] cols elements; y, dfdx [out] rows*cols elements.
+ *   y may equal x; dfdx may equal x; bias must not overlap an output.
+ *
+ * Backward: grad_in[r, c] = round(grad_out[r, c] * dfdx[r, c]) exactly as nfad_act_backward, and
+ *           grad_bias[c] = sum over r of the STORED (rounded) grad_in[r, c], accumulated in fp32
+ *           in a fixed order (so the result is reproducible run to run and does not depend on
+ *           pointer alignment): the rows are cut into chunks of consecutive rows, each chunk is
+ *           summed in row order, then the chunks' sums are added in order.  grad_bias is always fp32.
+ *   grad_out, dfdx [in], grad_in [out] rows*cols elements (grad_in may equal grad_out or dfdx);
+ *   grad_bias [out] cols floats (4-byte aligned); scratch: device memory of at least
+ *   nfad_bias_act_backward_scratch_bytes() bytes, 4-byte aligned, contents irrelevant before
+ *   and after; may be NULL when that size is 0.  Too small a scratch gives NFAD_E_SCRATCH.
+ *   rows == 0 gives grad_bias = 0.
+ *
+ * The 128-bit path needs cols to be a multiple of the packet (8 elements for the 16-bit
+ * types, 4 for fp32) and 16-byte aligned tensors; otherwise every element is handled one
+ * by one with identical results.  cols must be below 2^31 (NFAD_E_TOO_LARGE otherwise).
+ * The scratch size depends on the current device (its SM count decides how the rows are
+ * cut into chunks): ask for it with the device current that will run the call.
+ */
+NFAD_API int nfad_bias_act_forward(int kind, int dtype, const void* x, const void* bias, void* y, void* dfdx, size_t rows,
+                                   size_t cols, nfad_stream_t stream);
+NFAD_API int nfad_bias_act_backward(int kind, int dtype, const void* grad_out, const void* dfdx, void* grad_in,
+                                    float* grad_bias, void* scratch, size_t scratch_bytes, size_t rows, size_t cols,
+                                    nfad_stream_t stream);
+/* Bytes of scratch nfad_bias_act_backward needs on the current device; 0 on a bad dtype or when none is needed. */
+NFAD_API size_t nfad_bias_act_backward_scratch_bytes(int dtype, size_t rows, size_t cols);
+
+/*
  * Traffic probe (a measurement aid with no counterpart in the paper): moves
  * n_words 32-bit words per tensor through the same streaming kernel as the
  * activation pass, with a read/write mix of 1:1 (o0 = a), 1:2 (o0 = a, o1 = ~a)

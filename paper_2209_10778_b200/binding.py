@@ -30,6 +30,7 @@ EXPORTS = (
     "nfad_saved_bytes_per_element", "nfad_last_cuda_error", "nfad_status_string", "nfad_version",
     "nfad_probe_stream", "nfad_cmp_recompute_backward_noalloc",
     "nfad_seq_forward", "nfad_seq_backward", "nfad_ew_op",
+    "nfad_bias_act_forward", "nfad_bias_act_backward", "nfad_bias_act_backward_scratch_bytes",
 )
 OPCODES = {"add": 0, "mul": 1, "scale": 2, "add_const": 3, "exp": 4, "log1p": 5, "tanh": 6, "erf": 7, "softplus": 8,
            "sigmoid": 9, "half_one_plus_tanh": 10, "half_one_plus_erf": 11, "out": 12}
@@ -76,6 +77,12 @@ def load() -> ctypes.CDLL:
         lib.nfad_seq_backward.restype = ci
         lib.nfad_ew_op.argtypes = [ci, ci, ctypes.c_float, ci, vp, vp, vp, vp, vp, sz, vp]
         lib.nfad_ew_op.restype = ci
+        lib.nfad_bias_act_forward.argtypes = [ci, ci, vp, vp, vp, vp, sz, sz, vp]
+        lib.nfad_bias_act_forward.restype = ci
+        lib.nfad_bias_act_backward.argtypes = [ci, ci, vp, vp, vp, vp, vp, sz, sz, sz, vp]
+        lib.nfad_bias_act_backward.restype = ci
+        lib.nfad_bias_act_backward_scratch_bytes.argtypes = [ci, sz, sz]
+        lib.nfad_bias_act_backward_scratch_bytes.restype = sz
         lib.nfad_cmp_recompute_scratch_bytes.argtypes = [ci, ci, sz]
         lib.nfad_cmp_recompute_scratch_bytes.restype = sz
         lib.nfad_saved_bytes_per_element.argtypes = [ci, ci, ci]
@@ -178,6 +185,48 @@ def nfad_cmp_recompute_backward_noalloc(kind, grad_out: torch.Tensor, x: torch.T
                                                           _tensor(x, "x", grad_out), _tensor(grad_in, "grad_in", grad_out),
                                                           grad_out.numel(), _stream(grad_out)),
                "nfad_cmp_recompute_backward_noalloc")
+
+
+def _rows_cols(x: torch.Tensor, cols: int):
+    if cols <= 0 or x.numel() % cols:
+        raise ValueError("the tensor's size must be a multiple of the bias length")
+    return x.numel() // cols, cols
+
+
+def nfad_bias_act_forward(kind, x: torch.Tensor, bias: torch.Tensor, y: torch.Tensor, dfdx: torch.Tensor) -> None:
+    """x, y, dfdx: [..., cols] contiguous; bias: [cols] of the same dtype.  y = f(x + bias), dfdx = f'(x + bias)."""
+    px = _tensor(x, "x")
+    if bias.dtype != x.dtype or bias.device != x.device:
+        raise ValueError("bias must match x's dtype and device")
+    pb = _tensor(bias, "bias")
+    rows, cols = _rows_cols(x, bias.numel())
+    with torch.cuda.device(x.device):
+        _check(load().nfad_bias_act_forward(_kind(kind), _TORCH_TO_CODE[x.dtype], px, pb, _tensor(y, "y", x),
+                                            _tensor(dfdx, "dfdx", x), rows, cols, _stream(x)), "nfad_bias_act_forward")
+
+
+def nfad_bias_act_backward_scratch_bytes(dtype, rows: int, cols: int, device=None) -> int:
+    code = _TORCH_TO_CODE[dtype] if isinstance(dtype, torch.dtype) else DTYPES[dtype]
+    with torch.cuda.device(device if device is not None else torch.cuda.current_device()):
+        return int(load().nfad_bias_act_backward_scratch_bytes(code, rows, cols))
+
+
+def nfad_bias_act_backward(kind, grad_out: torch.Tensor, dfdx: torch.Tensor, grad_in: torch.Tensor, grad_bias: torch.Tensor,
+                           scratch: Optional[torch.Tensor]) -> None:
+    """grad_in = grad_out * dfdx; grad_bias (fp32, [cols]) = column sums of the stored grad_in.
+    scratch: a contiguous CUDA tensor of at least nfad_bias_act_backward_scratch_bytes bytes, or None if that is 0."""
+    pg = _tensor(grad_out, "grad_out")
+    if grad_bias.dtype != torch.float32 or not grad_bias.is_cuda or not grad_bias.is_contiguous():
+        raise TypeError("grad_bias must be a contiguous fp32 CUDA tensor")
+    rows, cols = _rows_cols(grad_out, grad_bias.numel())
+    if scratch is not None and (not scratch.is_cuda or not scratch.is_contiguous()):
+        raise TypeError("scratch must be a contiguous CUDA tensor")
+    sp = scratch.data_ptr() if scratch is not None else None
+    sb = scratch.numel() * scratch.element_size() if scratch is not None else 0
+    with torch.cuda.device(grad_out.device):
+        _check(load().nfad_bias_act_backward(_kind(kind), _TORCH_TO_CODE[grad_out.dtype], pg, _tensor(dfdx, "dfdx", grad_out),
+                                             _tensor(grad_in, "grad_in", grad_out), grad_bias.data_ptr(), sp, sb, rows, cols,
+                                             _stream(grad_out)), "nfad_bias_act_backward")
 
 
 def _ptr_array(tensors, name, like):

@@ -3,9 +3,10 @@
     python -m paper_2209_10778_b200.build          # rebuild if sources are newer
     python -m paper_2209_10778_b200.build --force
 
-Three translation units: the fp32-storage kernels are compiled with
+Five translation units: the fp32-storage kernels are compiled with
 floating-point contraction OFF (their compensated arithmetic depends on every
-fused multiply-add being written out), the 16-bit-storage kernels with it on,
+fused multiply-add being written out), the 16-bit-storage kernels and the run-time
+sequences with it on, the bias-gradient kernels (explicitly rounded intrinsics only),
 and the extern "C" boundary.  No fast-math, no flush-to-zero, IEEE division:
 subnormal inputs and results are part of the contract.
 """
@@ -28,6 +29,7 @@ UNITS = [
     ("nfad_kernels_f32.cu", ["-fmad=false"]),
     ("nfad_kernels_16.cu", ["-fmad=true"]),
     ("nfad_kernels_seq.cu", ["-fmad=true"]),
+    ("nfad_kernels_bias.cu", ["-fmad=false"]),
     ("nfad_api.cu", ["-fmad=false"]),
 ]
 

@@ -190,6 +190,97 @@ int nfad_probe_stream(int reads, int writes, const void* a, const void* b, void*
     return rc ? rc : run(op, 0, NFAD_F32, in, out, n_words, stream);
 }
 
+// ---- the pass fused with its producer's bias ----------------------------------------------
+
+static int check_shape(size_t rows, size_t cols, size_t* n)
+{
+    if (cols >= (size_t(1) << 31)) return NFAD_E_TOO_LARGE;
+    if (rows && cols > (~size_t(0) / 8) / rows) return NFAD_E_TOO_LARGE;     // rows * cols * element size must fit
+    *n = rows * cols;
+    return NFAD_OK;
+}
+
+int nfad_bias_act_forward(int kind, int dtype, const void* x, const void* bias, void* y, void* dfdx, size_t rows,
+                          size_t cols, nfad_stream_t stream)
+{
+    if (kind < 0 || kind > 3) return NFAD_E_KIND;
+    if (dtype < 0 || dtype > 2) return NFAD_E_DTYPE;
+    size_t n = 0;
+    int rc = check_shape(rows, cols, &n);
+    if (rc) return rc;
+    const void* in[1] = {x};
+    void* out[2] = {y, dfdx};
+    rc = check(kind, dtype, in, 1, out, 2, n);
+    if (rc || n == 0) return rc;
+    const size_t es = elem_size(dtype);
+    if (!bias) return NFAD_E_NULL;
+    if (reinterpret_cast<uintptr_t>(bias) % es) return NFAD_E_ALIGN;
+    if (overlaps(bias, y, cols * es, n * es) || overlaps(bias, dfdx, cols * es, n * es)) return NFAD_E_OVERLAP;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaError_t e = dtype == NFAD_F32 ? nfad::launch_bias_forward_f32(kind, x, bias, y, dfdx, rows, cols, st)
+                                      : nfad::launch_bias_forward_16(kind, dtype, x, bias, y, dfdx, rows, cols, st);
+    if (e != cudaSuccess) {
+        g_last_cuda_error = static_cast<int>(e);
+        return NFAD_E_CUDA;
+    }
+    return NFAD_OK;
+}
+
+size_t nfad_bias_act_backward_scratch_bytes(int dtype, size_t rows, size_t cols)
+{
+    if (dtype < 0 || dtype > 2) return 0;
+    size_t n = 0, bytes = 0;
+    if (check_shape(rows, cols, &n) != NFAD_OK || n == 0) return 0;
+    cudaError_t e = nfad::bias_backward_scratch(dtype, rows, cols, &bytes);
+    if (e != cudaSuccess) {
+        g_last_cuda_error = static_cast<int>(e);
+        return 0;
+    }
+    return bytes;
+}
+
+int nfad_bias_act_backward(int kind, int dtype, const void* grad_out, const void* dfdx, void* grad_in, float* grad_bias,
+                           void* scratch, size_t scratch_bytes, size_t rows, size_t cols, nfad_stream_t stream)
+{
+    if (kind < 0 || kind > 3) return NFAD_E_KIND;
+    if (dtype < 0 || dtype > 2) return NFAD_E_DTYPE;
+    size_t n = 0;
+    int rc = check_shape(rows, cols, &n);
+    if (rc) return rc;
+    if (cols == 0) return NFAD_OK;
+    const void* in[2] = {grad_out, dfdx};
+    void* out[1] = {grad_in};
+    rc = check(kind, dtype, in, 2, out, 1, n);
+    if (rc) return rc;
+    if (!grad_bias) return NFAD_E_NULL;
+    if (reinterpret_cast<uintptr_t>(grad_bias) % sizeof(float)) return NFAD_E_ALIGN;
+    const size_t es = elem_size(dtype), gb_bytes = cols * sizeof(float);
+    size_t need = 0;
+    cudaError_t e = cudaSuccess;
+    if (n) {
+        if (overlaps(grad_bias, grad_in, gb_bytes, n * es) || overlaps(grad_bias, grad_out, gb_bytes, n * es) ||
+            overlaps(grad_bias, dfdx, gb_bytes, n * es))
+            return NFAD_E_OVERLAP;
+        e = nfad::bias_backward_scratch(dtype, rows, cols, &need);
+        if (e == cudaSuccess && need) {
+            if (!scratch) return NFAD_E_NULL;
+            if (reinterpret_cast<uintptr_t>(scratch) % sizeof(float)) return NFAD_E_ALIGN;
+            if (scratch_bytes < need) return NFAD_E_SCRATCH;
+            if (overlaps(scratch, grad_in, need, n * es) || overlaps(scratch, grad_out, need, n * es) ||
+                overlaps(scratch, dfdx, need, n * es) || overlaps(scratch, grad_bias, need, gb_bytes))
+                return NFAD_E_OVERLAP;
+        }
+    }
+    if (e == cudaSuccess)
+        e = nfad::launch_bias_backward(dtype, grad_out, dfdx, grad_in, grad_bias, scratch, rows, cols,
+                                       static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) {
+        g_last_cuda_error = static_cast<int>(e);
+        return NFAD_E_CUDA;
+    }
+    return NFAD_OK;
+}
+
 int nfad_cmp_recompute_backward_noalloc(int kind, int dtype, const void* grad_out, const void* x, void* grad_in,
                                         size_t n, nfad_stream_t stream)
 {

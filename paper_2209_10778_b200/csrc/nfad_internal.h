@@ -35,4 +35,13 @@ cudaError_t launch_seq_forward(const SeqProgramHost& p, int dtype, const void* x
 cudaError_t launch_seq_backward(int dtype, const void* const* g, const void* const* d, int m, void* gin, size_t n, cudaStream_t st);
 cudaError_t launch_ew(int op, int backward, float c, int dtype, const void* const* in, void* const* out, size_t n, cudaStream_t st);
 
+// The pass fused with its producer's bias (nfad_bias.cuh).  x, y, d, g, gin: [rows, cols] row-major; bias: [cols].
+cudaError_t launch_bias_forward_f32(int kind, const void* x, const void* bias, void* y, void* d, size_t rows, size_t cols,
+                                    cudaStream_t st);
+cudaError_t launch_bias_forward_16(int kind, int dtype, const void* x, const void* bias, void* y, void* d, size_t rows,
+                                   size_t cols, cudaStream_t st);
+cudaError_t launch_bias_backward(int dtype, const void* g, const void* d, void* gin, float* grad_bias, void* scratch,
+                                 size_t rows, size_t cols, cudaStream_t st);
+cudaError_t bias_backward_scratch(int dtype, size_t rows, size_t cols, size_t* bytes);   // on the current device
+
 }  // namespace nfad

@@ -6,6 +6,7 @@
     python -m paper_2209_10778_b200.sweep --config stack      # 12 stacked GELU layers under three layouts
     python -m paper_2209_10778_b200.sweep --config probe      # plain 1:1 / 1:2 / 2:1 traffic through the same engine
     python -m paper_2209_10778_b200.sweep --config opbyop     # nested vs operator-by-operator back-propagation, measured
+    python -m paper_2209_10778_b200.sweep --config bias       # bias-add and bias gradient fused into the pass vs separate launches
 
 Each case launches one kernel `reps` times back to back between two CUDA events
 on the launching stream, after 3 warm-up launches; buffers are rotated so that
@@ -31,6 +32,7 @@ L2_BYTES = 126 * 1024 * 1024
 OPS = {
     "forward": (1, 2), "infer": (1, 1), "backward": (2, 1),
     "conv_backward": (2, 1), "recompute_backward": (2 + 1 + 1, 1 + 1),   # phase 1: x -> h; phase 2: g, x, h -> gin
+    "bias_forward": (1, 2), "bias_backward": (2, 1),                       # + cols elements of bias / cols floats: negligible
 }
 
 
@@ -57,9 +59,16 @@ def _make_sets(n, dtype, n_tensors, dev, std=1.0):
     return sets
 
 
-def time_case(kind: str, dtype: str, op: str, n: int, reps: int = 20, dev="cuda", std=1.0):
+def time_case(kind: str, dtype: str, op: str, n: int, reps: int = 20, dev="cuda", std=1.0, cols: int = 3072):
+    """cols: row length for the bias-fused calls (n must be a multiple of it)."""
     es = 4 if dtype == "f32" else 2
     sets = _make_sets(n, dtype, 5, dev, std)
+    if op.startswith("bias_"):
+        rows = n // cols
+        bias = W.normal(cols, dtype, 3, 0.5, dev)
+        gb = torch.empty(cols, dtype=torch.float32, device=dev)
+        nb = nfad.nfad_bias_act_backward_scratch_bytes(dtype, rows, cols)
+        bias_scratch = torch.empty(max(nb, 4), dtype=torch.uint8, device=dev) if nb else None
     for s in sets:
         nfad.nfad_act_forward(kind, s["x"], s["y"], s["d"])
     scratch = None
@@ -79,6 +88,10 @@ def time_case(kind: str, dtype: str, op: str, n: int, reps: int = 20, dev="cuda"
             nfad.nfad_cmp_conv_backward(kind, s["g"], s["x"], s["gin"])
         elif op == "recompute_backward":
             nfad.nfad_cmp_recompute_backward(kind, s["g"], s["x"], scratch[i % len(sets)], s["gin"])
+        elif op == "bias_forward":
+            nfad.nfad_bias_act_forward(kind, s["x"], bias, s["y"], s["d"])
+        elif op == "bias_backward":
+            nfad.nfad_bias_act_backward(kind, s["g"], s["d"], s["gin"], gb, bias_scratch)
         else:
             raise ValueError(op)
 
@@ -246,9 +259,77 @@ def run_stack(layers: int, n: int, dtype: str, kind: str, dev="cuda", reps: int 
     return out
 
 
+def run_bias(rows: int, cols: int, dtype: str, kinds, reps: int = 20, dev="cuda"):
+    """The pass with its producer's bias, fused (nfad_bias_act_*) against the same work as separate launches:
+    forward = a torch add that writes the pre-activation + nfad_act_forward; backward = nfad_act_backward + a torch
+    column sum (fp32 accumulate) over the stored grad_in.  Times are per forward / per backward."""
+    n = rows * cols
+    es = 4 if dtype == "f32" else 2
+    peak, src = _peak()
+    sets = _make_sets(n, dtype, 6, dev)
+    bias = W.normal(cols, dtype, 3, 0.5, dev)
+    gb = torch.empty(cols, dtype=torch.float32, device=dev)
+    nb = nfad.nfad_bias_act_backward_scratch_bytes(dtype, rows, cols)
+    scratch = torch.empty(max(nb, 4), dtype=torch.uint8, device=dev) if nb else None
+    for s in sets:
+        s["z"] = torch.empty_like(s["x"])
+
+    def timed(fn):
+        # `reps` launches replayed from one CUDA graph: at 12.6M elements a launch is ~15 us and the
+        # host (Python binding, torch dispatch) would otherwise be what is timed
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            for i in range(3):
+                fn(sets[i % len(sets)])
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            for i in range(reps):
+                fn(sets[(3 + i) % len(sets)])
+        graph.replay()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        graph.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / reps
+
+    out = []
+    for kind in kinds:
+        for s in sets:
+            nfad.nfad_bias_act_forward(kind, s["x"], bias, s["y"], s["d"])
+
+        def fwd_fused(s):
+            nfad.nfad_bias_act_forward(kind, s["x"], bias, s["y"], s["d"])
+
+        def fwd_split(s):
+            torch.add(s["x"].view(rows, cols), bias, out=s["z"].view(rows, cols))
+            nfad.nfad_act_forward(kind, s["z"], s["y"], s["d"])
+
+        def bwd_fused(s):
+            nfad.nfad_bias_act_backward(kind, s["g"], s["d"], s["gin"], gb, scratch)
+
+        def bwd_split(s):
+            nfad.nfad_act_backward(kind, s["g"], s["d"], s["gin"])
+            torch.sum(s["gin"].view(rows, cols), dim=0, dtype=torch.float32, out=gb)
+
+        for name, fn, tensors in (("forward fused", fwd_fused, 3), ("forward separate", fwd_split, 5),
+                                  ("backward fused", bwd_fused, 3), ("backward separate", bwd_split, 4)):
+            ms = timed(fn)
+            fused_bytes = 3 * es * n
+            out.append({"config": "bias", "kind": kind, "dtype": dtype, "rows": rows, "cols": cols, "case": name, "ms": ms,
+                        "tensor_passes": tensors, "GBps_of_fused_bytes": fused_bytes / (ms / 1e3) / 1e9,
+                        "frac_of_peak": fused_bytes / (ms / 1e3) / 1e9 / peak, "peak_GBps": peak, "peak_source": src})
+    return out
+
+
 def main(argv=None):
     ap = argparse.ArgumentParser()
-    ap.add_argument("--config", default=None, choices=[None, "sizes", "resnet50", "stack", "bert", "probe", "opbyop"])
+    ap.add_argument("--config", default=None, choices=[None, "sizes", "resnet50", "stack", "bert", "probe", "opbyop", "bias"])
+    ap.add_argument("--cols", type=int, default=3072)
     ap.add_argument("--n", type=int, default=100663296)
     ap.add_argument("--kinds", default="gelu_erf,gelu_tanh,swish,mish")
     ap.add_argument("--dtypes", default="bf16")
@@ -292,6 +373,11 @@ def main(argv=None):
         for dtype in dtypes:
             for r in run_opbyop(args.n, dtype, kinds):
                 print(json.dumps(r), flush=True)
+    elif args.config == "bias":
+        for dtype in dtypes:
+            for r in run_bias(args.n // args.cols, args.cols, dtype, kinds, args.reps):
+                print(json.dumps(r), flush=True)
+            torch.cuda.empty_cache()
     elif args.config == "stack":
         w = W.WORKLOADS["gelu_stack_12"]
         for r in run_stack(w.layers, w.numel(0), w.dtype, w.kinds[0]):

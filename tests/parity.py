@@ -47,6 +47,12 @@ def _fail_report(name, bad, x, got, want, err):
 
 def check_forward_fp32(kind: str, x_raw: np.ndarray, y: np.ndarray, d: np.ndarray, stats: dict | None = None):
     f, fp, cond = oracle.forward(kind, "f32", x_raw, want_cond=True)
+    check_forward_fp32_values(kind, x_raw, f, fp, cond, y, d, stats)
+
+
+def check_forward_fp32_values(kind: str, x_raw: np.ndarray, f: np.ndarray, fp: np.ndarray, cond: np.ndarray, y: np.ndarray,
+                              d: np.ndarray, stats: dict | None = None):
+    """x_raw: the point the activation was evaluated at; f, fp, cond: the oracle's values there."""
     xd = x_raw.astype(np.float64)
     # value
     ey = ulp.err_strict32(y, f)
@@ -76,11 +82,16 @@ def check_forward_fp32(kind: str, x_raw: np.ndarray, y: np.ndarray, d: np.ndarra
 def check_forward_16(kind: str, dtype: str, x_raw: np.ndarray, y_bits: np.ndarray, d_bits: np.ndarray,
                      stats: dict | None = None):
     f, fp = oracle.forward(kind, dtype, x_raw)
+    check_forward_16_values(kind, dtype, oracle.widen(dtype, x_raw), f, fp, y_bits, d_bits, stats)
+
+
+def check_forward_16_values(kind: str, dtype: str, xw: np.ndarray, f: np.ndarray, fp: np.ndarray, y_bits: np.ndarray,
+                            d_bits: np.ndarray, stats: dict | None = None):
+    """xw: the point the activation was evaluated at (fp64); f, fp: the oracle's unrounded values there."""
     want_y = oracle.round_to(dtype, f)
     want_d = oracle.round_to(dtype, fp)
     dy = ulp.ulp_distance16(y_bits, want_y)
     dd = ulp.ulp_distance16(d_bits, want_d)
-    xw = oracle.widen(dtype, x_raw)
     bad = (dy > 1) | ulp.is_nan16(y_bits, dtype)
     assert not bad.any(), _fail_report(f"{kind} {dtype} y", bad, xw, oracle.widen(dtype, y_bits), f, dy.astype(np.float64))
     badd = (dd > 1) | ulp.is_nan16(d_bits, dtype)
