@@ -33,6 +33,32 @@ class NestedActivation(torch.autograd.Function):
         return gin, None
 
 
+class NestedBiasActivation(torch.autograd.Function):
+    """y = f(x + bias) for x of shape [..., cols] and bias of shape [cols]: f'(x + bias) is the only saved tensor;
+    backward gives grad_x = grad_out * f' and grad_bias = its column sums, from one kernel."""
+
+    @staticmethod
+    def forward(ctx, x: torch.Tensor, bias: torch.Tensor, kind: str):
+        xc, bc = x.contiguous(), bias.contiguous()
+        y = torch.empty_like(xc)
+        d = torch.empty_like(xc)
+        nfad.nfad_bias_act_forward(kind, xc.view(-1), bc, y.view(-1), d.view(-1))
+        ctx.save_for_backward(d)
+        ctx.kind, ctx.cols, ctx.bias_dtype = kind, bc.numel(), bias.dtype
+        return y
+
+    @staticmethod
+    def backward(ctx, grad_out: torch.Tensor):
+        (d,) = ctx.saved_tensors
+        g = grad_out.contiguous()
+        gin = torch.empty_like(g)
+        gb = torch.empty(ctx.cols, dtype=torch.float32, device=g.device)
+        nbytes = nfad.nfad_bias_act_backward_scratch_bytes(g.dtype, g.numel() // ctx.cols, ctx.cols, g.device)
+        scratch = torch.empty(nbytes, dtype=torch.uint8, device=g.device) if nbytes else None
+        nfad.nfad_bias_act_backward(ctx.kind, g.view(-1), d.view(-1), gin.view(-1), gb, scratch)
+        return gin, gb.to(ctx.bias_dtype), None
+
+
 class ConventionalActivation(torch.autograd.Function):
     """The comparator that saves x and re-derives f'(x) in one fused backward kernel."""
 
@@ -70,6 +96,10 @@ class FadSequence(torch.autograd.Function):
         ds = ctx.saved_tensors
         gs = [g.contiguous().view(-1) for g in grad_outs]
         return sequence.backward_fused(gs, list(ds)).view(ctx.shape), None
+
+
+def bias_gelu(x, bias, approximate: str = "none"):
+    return NestedBiasActivation.apply(x, bias, "gelu_tanh" if approximate == "tanh" else "gelu_erf")
 
 
 def gelu(x, approximate: str = "none"):

@@ -277,7 +277,8 @@ NFAD_DEV Gate<Full> dual_half_one_plus_erf(const Dual<Full>& z)
     F2 sq = two_prod(za, za);
     ExpParts E = exp_parts_full(-sq.h, -sq.l); // exp(-za^2): the square is exact
     F2 a = f2_mul(half_erfcx_full(za), E.p);   // erfc(za)/2, without 2^n
-    float t0 = f2_value(f2_mul(E.p, kInvSqrtPi));   // its slope's magnitude at za, without 2^n
+    // its slope's magnitude at za, without 2^n: one rounding, of the leading product
+    float t0 = fmaf(E.p.h, kInvSqrtPi.h, fmaf(E.p.h, kInvSqrtPi.l, E.p.l * kInvSqrtPi.h));
     // first order in the low part of the argument: the value moves by -t0 zla,
     // the exponential by the factor (1 - 2 za zla)
     a.l = fmaf(-t0, zla, a.l);

@@ -198,10 +198,12 @@ NFAD_DEV F2 half_erfcx_full(float z)
     p = fmaf(p, q, -0.0334202126f);
     p = fmaf(p, q, 0.162647396f);
     p = fmaf(p, q, -0.360152066f);
-    // last Horner step c0 + q p without losing its rounding
-    F2 t = two_prod(p, q);
-    F2 s = two_sum(0.515540004f, t.h);
-    s.l += t.l;
+    // last Horner step c0 + q p without losing its rounding: the sum stays in [0.28, 1.07], so c0 - s.h is
+    // exact and a second fused multiply-add returns what the first one rounded away
+    const float c0 = 0.515540004f;
+    F2 s;
+    s.h = fmaf(p, q, c0);
+    s.l = fmaf(p, q, c0 - s.h);
     return f2_mul(s, r);
 }
 

@@ -225,3 +225,24 @@ def test_bert_ffn_shape_full_size(kind):
     # the bench workload's tensor, [32*128, 3072] bf16, every element against the oracle
     rows, cols = 32 * 128, 3072
     _run(kind, "bf16", rows, cols, 77, x_std=1.0)
+
+
+def test_autograd_wrapper_against_torch_double():
+    # the wrapper's gradients for x and the bias against torch's own autograd of gelu(x + b) in fp64
+    from paper_2209_10778_b200 import autograd as nfad_autograd
+    rows, cols = 96, 256
+    x = W.normal(rows * cols, "f32", 41, 1.5, DEV).view(4, rows // 4, cols).requires_grad_(True)
+    b = W.normal(cols, "f32", 42, 0.5, DEV).requires_grad_(True)
+    g = W.normal(rows * cols, "f32", 43, 1.0, DEV).view(4, rows // 4, cols)
+    for approx in ("none", "tanh"):
+        x.grad = b.grad = None
+        y = nfad_autograd.bias_gelu(x, b, approx)
+        y.backward(g)
+        x64 = x.detach().double().requires_grad_(True)
+        b64 = b.detach().double().requires_grad_(True)
+        y64 = torch.nn.functional.gelu(x64 + b64, approximate=approx)
+        y64.backward(g.double())
+        torch.cuda.synchronize()
+        assert torch.allclose(y.detach().double(), y64.detach(), rtol=1e-6, atol=1e-7)
+        assert torch.allclose(x.grad.double(), x64.grad, rtol=2e-6, atol=2e-6)
+        assert ((b.grad.double() - b64.grad).abs() <= 1e-5 * x64.grad.view(rows, cols).abs().sum(0) + 1e-6).all()
