@@ -265,7 +265,8 @@ NFAD_API int nfad_ew_op(int op, int backward, float c, int dtype, const void* in
  *           grad_bias[c] = sum over r of the STORED (rounded) grad_in[r, c], accumulated in fp32
  *           in a fixed order (so the result is reproducible run to run and does not depend on
  *           pointer alignment): the rows are cut into chunks of consecutive rows, each chunk is
- *           summed in row order, then the chunks' sums are added in order.  grad_bias is always fp32.
+ *           summed in row order, then the chunks' sums are added in a fixed order (32 runs of
+ *           consecutive chunks, then the runs).  grad_bias is always fp32.
  *   grad_out, dfdx [in], grad_in [out] rows*cols elements (grad_in may equal grad_out or dfdx);
  *   grad_bias [out] cols floats (4-byte aligned); scratch: device memory of at least
  *   nfad_bias_act_backward_scratch_bytes() bytes, 4-byte aligned, contents irrelevant before

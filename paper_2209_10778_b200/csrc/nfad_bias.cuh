@@ -73,7 +73,7 @@ struct BiasForwardArgs {
     void* d;
     size_t rows;
     size_t n;              // rows * cols
-    size_t work;           // strips * row chunks (vector path)
+    size_t work;           // row chunks (vector path)
     uint32_t cols;
     uint32_t row_packets;  // cols / V
     uint32_t strips;       // CTAs along a row
@@ -81,6 +81,22 @@ struct BiasForwardArgs {
 
 // z = x + b, one fp32 addition that the compiler may not merge into anything
 __device__ __forceinline__ float bias_sum(float x, float b) { return __fadd_rn(x, b); }
+
+template <class S, class K, class P>
+__device__ __forceinline__ void bias_forward_packet(const uint4& rx, const float (&vb)[S::kVec], uint4* y, uint4* d)
+{
+    constexpr int V = S::kVec;
+    float vx[V], vy[V], vd[V];
+    S::unpack(rx, vx);
+#pragma unroll
+    for (int e = 0; e < V; ++e) {
+        ActOut o = evaluate<K, P>(bias_sum(vx[e], vb[e]));
+        vy[e] = o.y;
+        vd[e] = o.dydx;
+    }
+    store_packet<true>(y, S::pack(vy));
+    store_packet<false>(d, S::pack(vd));
+}
 
 // Vector path: cols a multiple of the packet size and every pointer 16-byte aligned.
 template <class S, class K, class P>
@@ -95,32 +111,28 @@ __global__ void __launch_bounds__(kBiasMaxBlock, S::kMinBlocks) bias_forward_ker
     const uint4* x4 = static_cast<const uint4*>(a.x);
     uint4* y4 = static_cast<uint4*>(a.y);
     uint4* d4 = static_cast<uint4*>(a.d);
-    for (size_t w = blockIdx.x; w < a.work; w += gridDim.x) {
-        const uint32_t strip = uint32_t(w % a.strips);
-        const size_t r0 = (w / a.strips) * U;
-        const uint32_t cp = strip * blockDim.x + threadIdx.x;
-        if (cp >= a.row_packets) continue;
+    // grid: x = strip along the row (fastest, so neighbouring CTAs touch neighbouring memory), y = row chunk
+    const uint32_t cp = blockIdx.x * blockDim.x + threadIdx.x;
+    if (cp >= a.row_packets) return;
+    for (size_t chunk = blockIdx.y; chunk < a.work; chunk += gridDim.y) {
+        const size_t r0 = chunk * U;
         float vb[V];
         S::unpack(__ldg(static_cast<const uint4*>(a.bias) + cp), vb);
+        const size_t pk0 = r0 * a.row_packets + cp;
+        const uint32_t rp = a.row_packets;
         uint4 rx[U];
+        if (r0 + U <= a.rows) {                                        // whole tile: no predicates
 #pragma unroll
-        for (int u = 0; u < U; ++u)
-            if (r0 + u < a.rows) rx[u] = load_packet(x4 + (r0 + u) * a.row_packets + cp);
+            for (int u = 0; u < U; ++u) rx[u] = load_packet(x4 + pk0 + size_t(u) * rp);
 #pragma unroll
-        for (int u = 0; u < U; ++u) {
-            if (r0 + u < a.rows) {
-                float vx[V], vy[V], vd[V];
-                S::unpack(rx[u], vx);
+            for (int u = 0; u < U; ++u) bias_forward_packet<S, K, P>(rx[u], vb, y4 + pk0 + size_t(u) * rp, d4 + pk0 + size_t(u) * rp);
+        } else {
 #pragma unroll
-                for (int e = 0; e < V; ++e) {
-                    ActOut o = evaluate<K, P>(bias_sum(vx[e], vb[e]));
-                    vy[e] = o.y;
-                    vd[e] = o.dydx;
-                }
-                const size_t pk = (r0 + u) * a.row_packets + cp;
-                store_packet<true>(y4 + pk, S::pack(vy));
-                store_packet<false>(d4 + pk, S::pack(vd));
-            }
+            for (int u = 0; u < U; ++u)
+                if (r0 + u < a.rows) rx[u] = load_packet(x4 + pk0 + size_t(u) * rp);
+#pragma unroll
+            for (int u = 0; u < U; ++u)
+                if (r0 + u < a.rows) bias_forward_packet<S, K, P>(rx[u], vb, y4 + pk0 + size_t(u) * rp, d4 + pk0 + size_t(u) * rp);
         }
     }
 }
@@ -165,8 +177,9 @@ cudaError_t launch_bias_forward(const void* x, const void* bias, void* y, void* 
     a.row_packets = uint32_t(cols / V);
     const unsigned block = bias_block(a.row_packets);
     a.strips = (a.row_packets + block - 1) / block;
-    a.work = size_t(a.strips) * ((rows + kBiasRows - 1) / kBiasRows);
-    bias_launch_config(&cfg, attr, a.work < size_t(0x7fffffff) ? a.work : size_t(0x7fffffff), block, st, true);
+    a.work = (rows + kBiasRows - 1) / kBiasRows;
+    bias_launch_config(&cfg, attr, a.strips, block, st, true);
+    cfg.gridDim.y = (unsigned)(a.work < 65535 ? a.work : 65535);
     return cudaLaunchKernelEx(&cfg, bias_forward_kernel<S, K, P>, a);
 }
 
@@ -178,7 +191,6 @@ struct BiasBackwardArgs {
     void* gin;
     float* partial;          // [chunks][cols] sums, or grad_bias itself when chunks == 1
     size_t rows;
-    size_t work;             // strips * chunks (vector path)
     uint32_t cols;
     uint32_t row_packets;    // cols / V (vector path)
     uint32_t strips;
@@ -234,11 +246,10 @@ __global__ void __launch_bounds__(kBiasMaxBlock, 4) bias_backward_kernel(const B
     const uint4* g4 = static_cast<const uint4*>(a.g);
     const uint4* d4 = static_cast<const uint4*>(a.d);
     uint4* o4 = static_cast<uint4*>(a.gin);
-    for (size_t w = blockIdx.x; w < a.work; w += gridDim.x) {
-        const uint32_t strip = uint32_t(w % a.strips);
-        const size_t chunk = w / a.strips;
-        const uint32_t cp = strip * blockDim.x + threadIdx.x;
-        if (cp >= a.row_packets) continue;
+    const uint32_t cp = blockIdx.x * blockDim.x + threadIdx.x;     // grid: x = strip along the row, y = chunk of rows
+    if (cp >= a.row_packets) return;
+    {
+        const size_t chunk = blockIdx.y;
         const size_t r0 = chunk * a.chunk_rows;
         const size_t r1 = r0 + a.chunk_rows < a.rows ? r0 + a.chunk_rows : a.rows;
         float acc[V];
@@ -301,10 +312,11 @@ __global__ void __launch_bounds__(kBlock) bias_backward_scalar_kernel(const Bias
 
 // grad_bias[c] from partial[k][c], k < chunks, in a fixed order: the chunks are cut into kBiasGroups runs of
 // consecutive chunks, each run is summed in chunk order by one thread, and the runs' sums are added in run order.
-// A CTA takes 32 columns (one 128-byte line of every partial row) times the kBiasGroups runs.
-constexpr int kBiasGroups = kBlock / 32;
-static __global__ void __launch_bounds__(kBlock) bias_reduce_chunks_kernel(const float* partial, float* grad_bias, uint32_t chunks,
-                                                                           uint32_t cols)
+// A CTA takes 32 columns (one 128-byte line of every partial row) times the kBiasGroups runs; a thread's loads
+// are issued eight at a time before the first is used.
+constexpr int kBiasGroups = 32;
+static __global__ void __launch_bounds__(32 * kBiasGroups) bias_reduce_chunks_kernel(const float* partial, float* grad_bias,
+                                                                                     uint32_t chunks, uint32_t cols)
 {
     __shared__ float smem[kBiasGroups][32];
 #if NFAD_PDL
@@ -316,8 +328,16 @@ static __global__ void __launch_bounds__(kBlock) bias_reduce_chunks_kernel(const
     const uint32_t k0 = group * per;
     const uint32_t k1 = k0 + per < chunks ? k0 + per : chunks;
     float s = 0.0f;
-    if (col < cols)
-        for (uint32_t k = k0; k < k1; ++k) s = __fadd_rn(s, partial[size_t(k) * cols + col]);
+    if (col < cols) {
+        for (uint32_t k = k0; k < k1; k += 8) {
+            float v[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) v[j] = k + j < k1 ? partial[size_t(k + j) * cols + col] : 0.0f;
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+                if (k + j < k1) s = __fadd_rn(s, v[j]);
+        }
+    }
     smem[group][lane] = s;
     __syncthreads();
     if (group == 0 && col < cols) {
@@ -354,12 +374,12 @@ cudaError_t launch_bias_backward(const void* g, const void* d, void* gin, float*
     a.row_packets = uint32_t(cols / V);
     a.strips = p.strips;
     a.chunk_rows = p.chunk_rows;
-    a.work = size_t(p.strips) * p.chunks;
     const bool vec = cols % V == 0 && aligned16(g) && aligned16(d) && aligned16(gin);
     cudaLaunchConfig_t cfg;
     cudaLaunchAttribute attr[1];
     if (vec) {
-        bias_launch_config(&cfg, attr, a.work, p.block, st, true);
+        bias_launch_config(&cfg, attr, p.strips, p.block, st, true);
+        cfg.gridDim.y = p.chunks;
         e = cudaLaunchKernelEx(&cfg, bias_backward_kernel<S, kBf16>, a);
     } else {
         bias_launch_config(&cfg, attr, (cols + kBlock - 1) / kBlock, kBlock, st, false);
@@ -367,7 +387,7 @@ cudaError_t launch_bias_backward(const void* g, const void* d, void* gin, float*
         e = cudaLaunchKernelEx(&cfg, bias_backward_scalar_kernel<S, kBf16>, a);
     }
     if (e != cudaSuccess || p.chunks == 1) return e;
-    bias_launch_config(&cfg, attr, (cols + 31) / 32, kBlock, st, true);
+    bias_launch_config(&cfg, attr, (cols + 31) / 32, 32 * kBiasGroups, st, true);
     return cudaLaunchKernelEx(&cfg, bias_reduce_chunks_kernel, static_cast<const float*>(a.partial), grad_bias, p.chunks,
                               uint32_t(cols));
 }
