@@ -96,6 +96,21 @@ typedef void* nfad_stream_t;   /* a cudaStream_t */
 NFAD_API int nfad_act_forward(int kind, int dtype, const void* x, void* y, void* dfdx, size_t n, nfad_stream_t stream);
 
 /*
+ * Forward pass with the derivative held to the LITERAL 4-ulp bound for every input (fp32 storage
+ * only; any other dtype gives NFAD_E_DTYPE).  For x < 0, f' = h + x h' (Eq. 3 applied to f = x h) is
+ * a difference of two terms of similar size that changes sign, so arithmetic good to an fp32 ulp of
+ * the terms -- what nfad_act_forward guarantees there -- is not good to an fp32 ulp of f' near the
+ * sign change.  This entry point forms the two terms for x < 0 in fp64 and rounds their difference
+ * once: dfdx is within 4 fp32 ulp (in fact about one) of the exact f'(x) for every finite x, the
+ * neighbours of the sign change included; results below 2^-126 are rounded once to the subnormal
+ * grid.  y, and dfdx for x >= 0, are bit-identical to nfad_act_forward.  Same pointer, aliasing and
+ * stream rules.  Costs fp64 arithmetic on every element with x < 0 (see the measured rates).
+ * The 16-bit storage types need no such variant: there nfad_act_forward is within one ulp of the
+ * correctly rounded f' for every input.
+ */
+NFAD_API int nfad_act_forward_strict(int kind, int dtype, const void* x, void* y, void* dfdx, size_t n, nfad_stream_t stream);
+
+/*
  * Forward pass without the tangent (inference, or any pass that will not be
  * differentiated): the same chain of primitives, value parts only.
  *   x [in] n elements;  y [out] n elements (may equal x).

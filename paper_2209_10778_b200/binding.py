@@ -31,6 +31,7 @@ EXPORTS = (
     "nfad_probe_stream", "nfad_cmp_recompute_backward_noalloc",
     "nfad_seq_forward", "nfad_seq_backward", "nfad_ew_op",
     "nfad_bias_act_forward", "nfad_bias_act_backward", "nfad_bias_act_backward_scratch_bytes",
+    "nfad_act_forward_strict",
 )
 OPCODES = {"add": 0, "mul": 1, "scale": 2, "add_const": 3, "exp": 4, "log1p": 5, "tanh": 6, "erf": 7, "softplus": 8,
            "sigmoid": 9, "half_one_plus_tanh": 10, "half_one_plus_erf": 11, "out": 12}
@@ -65,6 +66,8 @@ def load() -> ctypes.CDLL:
         lib = ctypes.CDLL(LIB_PATH)
         vp, sz, ci = ctypes.c_void_p, ctypes.c_size_t, ctypes.c_int
         lib.nfad_act_forward.argtypes = [ci, ci, vp, vp, vp, sz, vp]
+        lib.nfad_act_forward_strict.argtypes = [ci, ci, vp, vp, vp, sz, vp]
+        lib.nfad_act_forward_strict.restype = ci
         lib.nfad_act_forward_infer.argtypes = [ci, ci, vp, vp, sz, vp]
         lib.nfad_act_backward.argtypes = [ci, ci, vp, vp, vp, sz, vp]
         lib.nfad_cmp_conv_backward.argtypes = [ci, ci, vp, vp, vp, sz, vp]
@@ -131,6 +134,14 @@ def nfad_act_forward(kind, x: torch.Tensor, y: torch.Tensor, dfdx: torch.Tensor)
     with torch.cuda.device(x.device):
         _check(load().nfad_act_forward(_kind(kind), _TORCH_TO_CODE[x.dtype], px, _tensor(y, "y", x),
                                        _tensor(dfdx, "dfdx", x), x.numel(), _stream(x)), "nfad_act_forward")
+
+
+def nfad_act_forward_strict(kind, x: torch.Tensor, y: torch.Tensor, dfdx: torch.Tensor) -> None:
+    """fp32 only: as nfad_act_forward, with f' within 4 fp32 ulp of itself for every input."""
+    px = _tensor(x, "x")
+    with torch.cuda.device(x.device):
+        _check(load().nfad_act_forward_strict(_kind(kind), _TORCH_TO_CODE[x.dtype], px, _tensor(y, "y", x),
+                                              _tensor(dfdx, "dfdx", x), x.numel(), _stream(x)), "nfad_act_forward_strict")
 
 
 def nfad_act_forward_infer(kind, x: torch.Tensor, y: torch.Tensor) -> None:

@@ -116,6 +116,15 @@ int nfad_act_forward(int kind, int dtype, const void* x, void* y, void* dfdx, si
     return rc ? rc : run(nfad::kOpForward, kind, dtype, in, out, n, stream);
 }
 
+int nfad_act_forward_strict(int kind, int dtype, const void* x, void* y, void* dfdx, size_t n, nfad_stream_t stream)
+{
+    if (dtype != NFAD_F32) return NFAD_E_DTYPE;
+    const void* in[1] = {x};
+    void* out[2] = {y, dfdx};
+    int rc = check(kind, dtype, in, 1, out, 2, n);
+    return rc ? rc : run(nfad::kOpForwardStrict, kind, dtype, in, out, n, stream);
+}
+
 int nfad_act_forward_infer(int kind, int dtype, const void* x, void* y, size_t n, nfad_stream_t stream)
 {
     const void* in[1] = {x};

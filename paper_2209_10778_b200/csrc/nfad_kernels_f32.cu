@@ -3,6 +3,7 @@
 // explicitly and must not have others introduced by contraction.
 #include "nfad_bias.cuh"
 #include "nfad_dispatch.cuh"
+#include "nfad_strict.cuh"
 
 namespace nfad {
 
@@ -11,6 +12,15 @@ cudaError_t launch_f32(OpCode op, int kind, const void* const* in, void* const* 
     if (op == kOpProbe11) return launch_stream<StoreF32, ProbeOp<1, 1>>(in, out, n, st);
     if (op == kOpProbe12) return launch_stream<StoreF32, ProbeOp<1, 2>>(in, out, n, st);
     if (op == kOpProbe21) return launch_stream<StoreF32, ProbeOp<2, 1>>(in, out, n, st);
+    if (op == kOpForwardStrict) {
+        switch (kind) {
+        case kGeluErf:  return launch_stream<StoreF32, ForwardStrictOp<GeluErf>>(in, out, n, st);
+        case kGeluTanh: return launch_stream<StoreF32, ForwardStrictOp<GeluTanh>>(in, out, n, st);
+        case kSwish:    return launch_stream<StoreF32, ForwardStrictOp<Swish>>(in, out, n, st);
+        case kMish:     return launch_stream<StoreF32, ForwardStrictOp<Mish>>(in, out, n, st);
+        }
+        return cudaErrorInvalidValue;
+    }
     return dispatch_kind<StoreF32, Full, false>(op, kind, in, out, n, st);
 }
 

@@ -32,6 +32,7 @@ L2_BYTES = 126 * 1024 * 1024
 OPS = {
     "forward": (1, 2), "infer": (1, 1), "backward": (2, 1),
     "conv_backward": (2, 1), "recompute_backward": (2 + 1 + 1, 1 + 1),   # phase 1: x -> h; phase 2: g, x, h -> gin
+    "forward_strict": (1, 2),                                              # fp32 storage only
     "bias_forward": (1, 2), "bias_backward": (2, 1),                       # + cols elements of bias / cols floats: negligible
 }
 
@@ -80,6 +81,8 @@ def time_case(kind: str, dtype: str, op: str, n: int, reps: int = 20, dev="cuda"
         s = sets[i % len(sets)]
         if op == "forward":
             nfad.nfad_act_forward(kind, s["x"], s["y"], s["d"])
+        elif op == "forward_strict":
+            nfad.nfad_act_forward_strict(kind, s["x"], s["y"], s["d"])
         elif op == "infer":
             nfad.nfad_act_forward_infer(kind, s["x"], s["y"])
         elif op == "backward":

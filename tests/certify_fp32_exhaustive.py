@@ -1,6 +1,6 @@
 """Exhaustive certification of the fp32-storage forward kernels (not collected by pytest: run by hand).
 
-    python tests/certify_fp32_exhaustive.py [kind,kind,...]
+    python tests/certify_fp32_exhaustive.py [kind,kind,...] [--strict]
 
 Every fp32 bit pattern with |x| <= 130 (2 x 1.12e9 values per kind; beyond that every kind is
 saturated) goes through nfad_act_forward on cuda:0 and is compared with the fp64 oracle in the
@@ -8,6 +8,8 @@ metrics of tests/parity.py.  Prints, per kind, the worst value error in ulp, the
 derivative error in the gate's metric (strict for x >= 0, scaled by |h| + |x h'| for x < 0),
 the worst subnormal-result errors in units of 2^-149 and the count of non-finite outputs, and
 writes them to gpurun_out/exhaustive_f32.json.  About three minutes per kind on a 16-core host.
+With --strict the inputs go through nfad_act_forward_strict instead and the derivative is measured in
+strict ulp of f' itself for every x (no scaling); the results go to gpurun_out/exhaustive_f32_strict.json.
 """
 import json
 import os
@@ -23,7 +25,9 @@ sys.path.insert(0, os.path.join(ROOT, 'tests'))
 import oracle, ulp
 from paper_2209_10778_b200 import binding as nfad
 oracle.set_threads(oracle.max_threads())
-kinds = sys.argv[1].split(',') if len(sys.argv) > 1 else ['gelu_erf','gelu_tanh','swish','mish']
+STRICT = '--strict' in sys.argv
+args = [a for a in sys.argv[1:] if not a.startswith('--')]
+kinds = args[0].split(',') if args else ['gelu_erf','gelu_tanh','swish','mish']
 hi_bits = int(np.float32(130.0).view(np.uint32))
 CH = 1 << 25
 res = {}
@@ -37,7 +41,7 @@ for kind in kinds:
             x = (bits & 0xFFFFFFFF).to(torch.int64)
             x = torch.where(x >= 2**31, x - 2**32, x).to(torch.int32).view(torch.float32).contiguous()
             y = torch.empty_like(x); d = torch.empty_like(x)
-            nfad.nfad_act_forward(kind, x, y, d)
+            (nfad.nfad_act_forward_strict if STRICT else nfad.nfad_act_forward)(kind, x, y, d)
             torch.cuda.synchronize()
             xh, yh, dh = x.cpu().numpy(), y.cpu().numpy(), d.cpu().numpy()
             f, fp, T = oracle.forward(kind, 'f32', xh, want_cond=True)
@@ -46,8 +50,8 @@ for kind in kinds:
             ey = np.abs(yh.astype(np.float64) - f) / u32(f)
             es = np.abs(dh.astype(np.float64) - fp) / u32(fp)
             ec = np.abs(dh.astype(np.float64) - fp) / u32(np.maximum(T, np.abs(fp)))
-            gate = np.where(xh >= 0, es, ec)
-            suby = np.abs(f) < 2.0**-126; subd = (np.abs(fp) < 2.0**-126) & (T < 2.0**-100)
+            gate = es if STRICT else np.where(xh >= 0, es, ec)
+            suby = np.abs(f) < 2.0**-126; subd = (np.abs(fp) < 2.0**-126) & ((T < 2.0**-100) | STRICT)
             ny = np.where(suby, 0, ey); nd = np.where(subd, 0, gate)
             i = int(ny.argmax()); j = int(nd.argmax())
             if ny[i] > worst['y']: worst['y'] = float(ny[i]); worst['y_x'] = float(xh[i])
@@ -60,4 +64,4 @@ for kind in kinds:
     res[kind] = worst
     print(kind, json.dumps(worst), flush=True)
 os.makedirs(os.path.join(ROOT, 'gpurun_out'), exist_ok=True)
-json.dump(res, open(os.path.join(ROOT, 'gpurun_out', 'exhaustive_f32.json'), 'w'))
+json.dump(res, open(os.path.join(ROOT, 'gpurun_out', 'exhaustive_f32_strict.json' if STRICT else 'exhaustive_f32.json'), 'w'))
