@@ -247,22 +247,46 @@ def run_ours(args, w):
             for i in range(period):
                 step(i, False)
 
+    def group_launches(j: int, kind: str, first: int, count: int, backward: bool):
+        for i in range(first, first + count):
+            if backward:
+                b = sets[(len(kinds) * i + j + half) % n_sets]
+                nfad.nfad_act_backward(kind, b["g"], b["d"], b["gin"])
+            else:
+                a = sets[(len(kinds) * i + j) % n_sets]
+                nfad.nfad_act_forward(kind, a["x"], a["y"], a["d"])
+
+    # The same period of steps with its launches reordered kernel by kernel (all forwards of the first
+    # kind, all its backwards, then the next kind), each run captured in a graph of its own: the
+    # launches of a step are independent of one another, so this is the same work on the same buffers,
+    # and one event pair around a replay brackets `period` back-to-back launches of ONE kernel with
+    # neither the host's launch rate nor per-launch event latency in the figure.
+    group_graphs = None
+    if graph is not None:
+        group_graphs = []
+        for j, kind in enumerate(kinds):
+            pair = []
+            for backward in (False, True):
+                gg = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(gg):
+                    group_launches(j, kind, 0, period, backward)
+                pair.append(gg)
+            group_graphs.append(pair)
+
     def step_group(first: int, count: int):
-        """`count` whole steps with their launches reordered kernel by kernel (all forwards of the
-        first kind, all its backwards, then the next kind): the launches of a step are independent of
-        one another, so this is the same work on the same buffers, and it lets ONE event pair bracket
-        `count` back-to-back launches of one kernel -- the launch and event latency (5-7 us, as much
-        as a third of a 15 us kernel) is then paid once per group instead of once per launch."""
+        """`count` whole steps, kernel-major (see above); `first` is a multiple of the period when graphs are used."""
         for j, kind in enumerate(kinds):
             e0, e1, e2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
             e0.record()
-            for i in range(first, first + count):
-                a = sets[(len(kinds) * i + j) % n_sets]
-                nfad.nfad_act_forward(kind, a["x"], a["y"], a["d"])
+            if group_graphs is not None and count == period:
+                group_graphs[j][0].replay()
+            else:
+                group_launches(j, kind, first, count, False)
             e1.record()
-            for i in range(first, first + count):
-                b = sets[(len(kinds) * i + j + half) % n_sets]
-                nfad.nfad_act_backward(kind, b["g"], b["d"], b["gin"])
+            if group_graphs is not None and count == period:
+                group_graphs[j][1].replay()
+            else:
+                group_launches(j, kind, first, count, True)
             e2.record()
             if j == 0:
                 ev["fwd"].append((e0, e1, count))
@@ -315,8 +339,9 @@ def run_ours(args, w):
         sampler.stop()
     ms = ranks.max_over_ranks(wd, ms, dev)
 
-    timing_source = ("one event pair around the last %d steps' launches of this kernel, issued back to back "
-                     "at the end of the timed region" % min(args.steps, period))
+    timing_source = ("one event pair around the last %d steps' launches of this kernel, %s back to back "
+                     "at the end of the timed region" % (min(args.steps, period),
+                                                         "replayed from a graph" if graph is not None and args.steps >= period else "issued"))
     src = ev
     fwd_ms = statistics.mean(a.elapsed_time(b) / c for a, b, c in src["fwd"]) if src["fwd"] else None
     bwd_ms = statistics.mean(a.elapsed_time(b) / c for a, b, c in src["bwd"]) if src["bwd"] else None
