@@ -119,8 +119,37 @@ def _tensor(t: torch.Tensor, name: str, like: Optional[torch.Tensor] = None) -> 
     return t.data_ptr()
 
 
+_raw_stream = getattr(torch._C, "_cuda_getCurrentRawStream", None)
+
+
 def _stream(t: torch.Tensor) -> int:
+    """The current stream of the tensor's device, as a cudaStream_t."""
+    if _raw_stream is not None:
+        idx = t.device.index
+        return _raw_stream(idx if idx is not None else torch.cuda.current_device())
     return torch.cuda.current_stream(t.device).cuda_stream
+
+
+class _on_device:
+    """Makes the tensor's device current for the call; a no-op (two integer reads) when it already is --
+    the common case, and the one where the generic guard's cost would show in every small launch."""
+    __slots__ = ("idx", "prev")
+
+    def __init__(self, dev: torch.device):
+        self.idx = dev.index
+        self.prev = None
+
+    def __enter__(self):
+        cur = torch.cuda.current_device()
+        if self.idx is not None and self.idx != cur:
+            self.prev = cur
+            torch.cuda.set_device(self.idx)
+        return self
+
+    def __exit__(self, *exc):
+        if self.prev is not None:
+            torch.cuda.set_device(self.prev)
+        return False
 
 
 def _check(rc: int, where: str) -> None:
@@ -131,7 +160,7 @@ def _check(rc: int, where: str) -> None:
 def nfad_act_forward(kind, x: torch.Tensor, y: torch.Tensor, dfdx: torch.Tensor) -> None:
     """x -> (y = f(x), dfdx = f'(x)), one kernel on the current stream."""
     px = _tensor(x, "x")
-    with torch.cuda.device(x.device):
+    with _on_device(x.device):
         _check(load().nfad_act_forward(_kind(kind), _TORCH_TO_CODE[x.dtype], px, _tensor(y, "y", x),
                                        _tensor(dfdx, "dfdx", x), x.numel(), _stream(x)), "nfad_act_forward")
 
@@ -139,14 +168,14 @@ def nfad_act_forward(kind, x: torch.Tensor, y: torch.Tensor, dfdx: torch.Tensor)
 def nfad_act_forward_strict(kind, x: torch.Tensor, y: torch.Tensor, dfdx: torch.Tensor) -> None:
     """fp32 only: as nfad_act_forward, with f' within 4 fp32 ulp of itself for every input."""
     px = _tensor(x, "x")
-    with torch.cuda.device(x.device):
+    with _on_device(x.device):
         _check(load().nfad_act_forward_strict(_kind(kind), _TORCH_TO_CODE[x.dtype], px, _tensor(y, "y", x),
                                               _tensor(dfdx, "dfdx", x), x.numel(), _stream(x)), "nfad_act_forward_strict")
 
 
 def nfad_act_forward_infer(kind, x: torch.Tensor, y: torch.Tensor) -> None:
     px = _tensor(x, "x")
-    with torch.cuda.device(x.device):
+    with _on_device(x.device):
         _check(load().nfad_act_forward_infer(_kind(kind), _TORCH_TO_CODE[x.dtype], px, _tensor(y, "y", x),
                                              x.numel(), _stream(x)), "nfad_act_forward_infer")
 
@@ -154,7 +183,7 @@ def nfad_act_forward_infer(kind, x: torch.Tensor, y: torch.Tensor) -> None:
 def nfad_act_backward(kind, grad_out: torch.Tensor, dfdx: torch.Tensor, grad_in: torch.Tensor) -> None:
     """grad_in = grad_out * dfdx (one rounding)."""
     pg = _tensor(grad_out, "grad_out")
-    with torch.cuda.device(grad_out.device):
+    with _on_device(grad_out.device):
         _check(load().nfad_act_backward(_kind(kind), _TORCH_TO_CODE[grad_out.dtype], pg, _tensor(dfdx, "dfdx", grad_out),
                                         _tensor(grad_in, "grad_in", grad_out), grad_out.numel(), _stream(grad_out)),
                "nfad_act_backward")
@@ -162,7 +191,7 @@ def nfad_act_backward(kind, grad_out: torch.Tensor, dfdx: torch.Tensor, grad_in:
 
 def nfad_cmp_conv_backward(kind, grad_out: torch.Tensor, x: torch.Tensor, grad_in: torch.Tensor) -> None:
     pg = _tensor(grad_out, "grad_out")
-    with torch.cuda.device(grad_out.device):
+    with _on_device(grad_out.device):
         _check(load().nfad_cmp_conv_backward(_kind(kind), _TORCH_TO_CODE[grad_out.dtype], pg, _tensor(x, "x", grad_out),
                                              _tensor(grad_in, "grad_in", grad_out), grad_out.numel(), _stream(grad_out)),
                "nfad_cmp_conv_backward")
@@ -179,7 +208,7 @@ def nfad_cmp_recompute_backward(kind, grad_out: torch.Tensor, x: torch.Tensor, s
     pg = _tensor(grad_out, "grad_out")
     if not scratch.is_cuda or not scratch.is_contiguous():
         raise TypeError("scratch must be a contiguous CUDA tensor")
-    with torch.cuda.device(grad_out.device):
+    with _on_device(grad_out.device):
         _check(load().nfad_cmp_recompute_backward(_kind(kind), _TORCH_TO_CODE[grad_out.dtype], pg, _tensor(x, "x", grad_out),
                                                   scratch.data_ptr(), scratch.numel() * scratch.element_size(),
                                                   _tensor(grad_in, "grad_in", grad_out), grad_out.numel(),
@@ -191,7 +220,7 @@ def nfad_cmp_recompute_backward_noalloc(kind, grad_out: torch.Tensor, x: torch.T
     cannot allocate device memory where they stand.  At most NOALLOC_SCRATCH_BYTES per tensor;
     calls on one device share the array, so calls that may overlap on the GPU must be serialised."""
     pg = _tensor(grad_out, "grad_out")
-    with torch.cuda.device(grad_out.device):
+    with _on_device(grad_out.device):
         _check(load().nfad_cmp_recompute_backward_noalloc(_kind(kind), _TORCH_TO_CODE[grad_out.dtype], pg,
                                                           _tensor(x, "x", grad_out), _tensor(grad_in, "grad_in", grad_out),
                                                           grad_out.numel(), _stream(grad_out)),
@@ -211,7 +240,7 @@ def nfad_bias_act_forward(kind, x: torch.Tensor, bias: torch.Tensor, y: torch.Te
         raise ValueError("bias must match x's dtype and device")
     pb = _tensor(bias, "bias")
     rows, cols = _rows_cols(x, bias.numel())
-    with torch.cuda.device(x.device):
+    with _on_device(x.device):
         _check(load().nfad_bias_act_forward(_kind(kind), _TORCH_TO_CODE[x.dtype], px, pb, _tensor(y, "y", x),
                                             _tensor(dfdx, "dfdx", x), rows, cols, _stream(x)), "nfad_bias_act_forward")
 
@@ -234,7 +263,7 @@ def nfad_bias_act_backward(kind, grad_out: torch.Tensor, dfdx: torch.Tensor, gra
         raise TypeError("scratch must be a contiguous CUDA tensor")
     sp = scratch.data_ptr() if scratch is not None else None
     sb = scratch.numel() * scratch.element_size() if scratch is not None else 0
-    with torch.cuda.device(grad_out.device):
+    with _on_device(grad_out.device):
         _check(load().nfad_bias_act_backward(_kind(kind), _TORCH_TO_CODE[grad_out.dtype], pg, _tensor(dfdx, "dfdx", grad_out),
                                              _tensor(grad_in, "grad_in", grad_out), grad_bias.data_ptr(), sp, sb, rows, cols,
                                              _stream(grad_out)), "nfad_bias_act_backward")
@@ -260,7 +289,7 @@ def nfad_seq_forward(program, x: torch.Tensor, ys, dfdxs) -> None:
     px = _tensor(x, "x")
     if len(ys) != len(dfdxs):
         raise ValueError("ys and dfdxs must have the same length")
-    with torch.cuda.device(x.device):
+    with _on_device(x.device):
         _check(load().nfad_seq_forward(ops, len(program), _TORCH_TO_CODE[x.dtype], px, _ptr_array(ys, "y", x),
                                        _ptr_array(dfdxs, "dfdx", x), len(ys), x.numel(), _stream(x)), "nfad_seq_forward")
 
@@ -270,7 +299,7 @@ def nfad_seq_backward(grad_outs, dfdxs, grad_in: torch.Tensor) -> None:
     pg = _tensor(grad_in, "grad_in")
     if len(grad_outs) != len(dfdxs):
         raise ValueError("grad_outs and dfdxs must have the same length")
-    with torch.cuda.device(grad_in.device):
+    with _on_device(grad_in.device):
         _check(load().nfad_seq_backward(_TORCH_TO_CODE[grad_in.dtype], _ptr_array(grad_outs, "grad_out", grad_in),
                                         _ptr_array(dfdxs, "dfdx", grad_in), len(grad_outs), pg, grad_in.numel(),
                                         _stream(grad_in)), "nfad_seq_backward")
@@ -281,7 +310,7 @@ def nfad_ew_op(op, backward: bool, c: float, in0: torch.Tensor, in1, in2, out0: 
     p0 = _tensor(in0, "in0")
     code = OPCODES[op] if isinstance(op, str) else int(op)
     opt = lambda t, name: _tensor(t, name, in0) if t is not None else None
-    with torch.cuda.device(in0.device):
+    with _on_device(in0.device):
         _check(load().nfad_ew_op(code, 1 if backward else 0, float(c), _TORCH_TO_CODE[in0.dtype], p0, opt(in1, "in1"),
                                  opt(in2, "in2"), _tensor(out0, "out0", in0), opt(out1, "out1"), in0.numel(), _stream(in0)),
                "nfad_ew_op")
@@ -301,7 +330,7 @@ def nfad_probe_stream(reads: int, writes: int, a: torch.Tensor, b, o0: torch.Ten
     pa = _tensor(a, "a")
     if a.dtype != torch.float32:
         raise TypeError("the probe takes float32 tensors")
-    with torch.cuda.device(a.device):
+    with _on_device(a.device):
         _check(load().nfad_probe_stream(int(reads), int(writes), pa, _tensor(b, "b", a) if b is not None else None,
                                         _tensor(o0, "o0", a), _tensor(o1, "o1", a) if o1 is not None else None,
                                         a.numel(), _stream(a)), "nfad_probe_stream")

@@ -246,3 +246,9 @@ def test_autograd_wrapper_against_torch_double():
         assert torch.allclose(y.detach().double(), y64.detach(), rtol=1e-6, atol=1e-7)
         assert torch.allclose(x.grad.double(), x64.grad, rtol=2e-6, atol=2e-6)
         assert ((b.grad.double() - b64.grad).abs() <= 1e-5 * x64.grad.view(rows, cols).abs().sum(0) + 1e-6).all()
+
+
+def test_tall_narrow_tensor_covers_the_row_chunk_loop():
+    # more row chunks than one grid dimension holds (rows / 4 > 65535): the forward kernel's chunk loop, and a backward
+    # whose strips are narrower than one warp-wide access
+    _run("swish", "bf16", 300000, 64, 55)
