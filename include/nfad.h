@@ -308,6 +308,10 @@ NFAD_API size_t nfad_bias_act_backward_scratch_bytes(int dtype, size_t rows, siz
  * activation pass, with a read/write mix of 1:1 (o0 = a), 1:2 (o0 = a, o1 = ~a)
  * or 2:1 (o0 = a ^ b), so that the bandwidth a given mix can reach on the device
  * is known beside the activation kernels' numbers.  Unused tensors may be NULL.
+ * Two one-sided mixes measure the read and the write ceiling alone: 1:0 reads a and
+ * writes nothing (o0 is a one-word sink that is only written if a checksum of the data
+ * matches a fixed constant), 0:1 writes a fixed pattern to o0; both need a 16-byte
+ * aligned tensor of a multiple of 4 words (NFAD_E_ALIGN otherwise).
  * Any other mix gives NFAD_E_LAYOUT.  Same pointer, aliasing and stream rules as above.
  */
 NFAD_API int nfad_probe_stream(int reads, int writes, const void* a, const void* b, void* o0, void* o1, size_t n_words,

@@ -325,15 +325,25 @@ def nfad_saved_bytes_per_element(kind, dtype, layout) -> int:
     return rc
 
 
-def nfad_probe_stream(reads: int, writes: int, a: torch.Tensor, b, o0: torch.Tensor, o1) -> None:
-    """Traffic probe over fp32 tensors: 1:1 (o0 = a), 1:2 (o0 = a, o1 = ~a) or 2:1 (o0 = a ^ b)."""
-    pa = _tensor(a, "a")
-    if a.dtype != torch.float32:
+def nfad_probe_stream(reads: int, writes: int, a, b, o0: torch.Tensor, o1) -> None:
+    """Traffic probe over fp32 tensors: 1:1 (o0 = a), 1:2 (o0 = a, o1 = ~a), 2:1 (o0 = a ^ b),
+    1:0 (reads a; o0 is a sink of at least one word) or 0:1 (writes o0; a is None)."""
+    main = a if a is not None else o0
+    pm = _tensor(main, "a" if a is not None else "o0")
+    if main.dtype != torch.float32:
         raise TypeError("the probe takes float32 tensors")
-    with _on_device(a.device):
-        _check(load().nfad_probe_stream(int(reads), int(writes), pa, _tensor(b, "b", a) if b is not None else None,
-                                        _tensor(o0, "o0", a), _tensor(o1, "o1", a) if o1 is not None else None,
-                                        a.numel(), _stream(a)), "nfad_probe_stream")
+    one_sided = int(writes) == 0 or int(reads) == 0
+    with _on_device(main.device):
+        if one_sided:
+            po = _tensor(o0, "o0")
+            if o0.dtype != torch.float32 or o0.numel() < 1 or o0.device != main.device:
+                raise ValueError("o0 must be a float32 tensor on the same device")
+            _check(load().nfad_probe_stream(int(reads), int(writes), pm if a is not None else None, None, po, None,
+                                            main.numel(), _stream(main)), "nfad_probe_stream")
+        else:
+            _check(load().nfad_probe_stream(int(reads), int(writes), pm, _tensor(b, "b", a) if b is not None else None,
+                                            _tensor(o0, "o0", a), _tensor(o1, "o1", a) if o1 is not None else None,
+                                            a.numel(), _stream(a)), "nfad_probe_stream")
 
 
 def nfad_version() -> str:

@@ -192,7 +192,20 @@ int nfad_probe_stream(int reads, int writes, const void* a, const void* b, void*
     if (reads == 1 && writes == 1) op = nfad::kOpProbe11;
     else if (reads == 1 && writes == 2) op = nfad::kOpProbe12;
     else if (reads == 2 && writes == 1) op = nfad::kOpProbe21;
+    else if (reads == 1 && writes == 0) op = nfad::kOpProbe10;
+    else if (reads == 0 && writes == 1) op = nfad::kOpProbe01;
     else return NFAD_E_LAYOUT;
+    if (writes == 0 || reads == 0) {
+        // one-sided probes: whole 16-byte packets only; o0 is a one-word sink for the read probe
+        if (n_words == 0) return NFAD_OK;
+        if (!o0 || (reads && !a)) return NFAD_E_NULL;
+        const void* p = reads ? a : o0;
+        if ((reinterpret_cast<uintptr_t>(p) & 15u) || (reinterpret_cast<uintptr_t>(o0) & 3u) || (n_words & 3u)) return NFAD_E_ALIGN;
+        if (reads && overlaps(a, o0, n_words * 4, 4)) return NFAD_E_OVERLAP;
+        const void* in1[1] = {a};
+        void* out1[1] = {o0};
+        return run(op, 0, NFAD_F32, in1, out1, n_words, stream);
+    }
     const void* in[2] = {a, b};
     void* out[2] = {o0, o1};
     int rc = check(0, NFAD_F32, in, reads, out, writes, n_words);

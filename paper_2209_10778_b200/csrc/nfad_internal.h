@@ -20,8 +20,10 @@ enum DType { kF32 = 0, kBF16 = 1, kF16 = 2 };
 //   kOpRecompute2     in {g, x, h}      out {gin}
 //   kOpProbe11/12/21  in {a[, b]}       out {o0[, o1]}   (traffic probes: fp32 storage only)
 //   kOpForwardStrict  in {x}            out {y, dfdx}    (fp32 storage only)
+//   kOpProbe10        in {a}            out {sink}       (read-only probe; sink: one word, written only on a checksum match)
+//   kOpProbe01        in {}             out {o0}         (write-only probe)
 enum OpCode { kOpForward, kOpForwardInfer, kOpBackward, kOpConvBackward, kOpRecompute1, kOpRecompute2,
-              kOpProbe11, kOpProbe12, kOpProbe21, kOpForwardStrict };
+              kOpProbe11, kOpProbe12, kOpProbe21, kOpForwardStrict, kOpProbe10, kOpProbe01 };
 
 cudaError_t launch_f32(OpCode op, int kind, const void* const* in, void* const* out, size_t n, cudaStream_t st);
 cudaError_t launch_16(OpCode op, int kind, int dtype, const void* const* in, void* const* out, size_t n, cudaStream_t st);
