@@ -303,6 +303,41 @@ NFAD_API int nfad_bias_act_backward(int kind, int dtype, const void* grad_out, c
 NFAD_API size_t nfad_bias_act_backward_scratch_bytes(int dtype, size_t rows, size_t cols);
 
 /*
+ * The whole pass for tensors that live in HOST memory (no counterpart in the paper: a service entry
+ * point for callers whose activations are kept off the device, and the end-to-end form of the pass
+ * that the benchmark times).  Forward and backward of one batch:
+ *   x_host, grad_out_host [in, host]   n elements each
+ *   y_host, grad_in_host  [out, host]  n elements each: y = f(x), grad_in = round(grad_out * f'(x))
+ *   dfdx_host             [out, host]  n elements or NULL: the saved tensor, if the caller wants it
+ * with exactly the arithmetic of nfad_act_forward followed by nfad_act_backward (bit-identical
+ * results).  The batch is cut into chunks that move through a three-stage pipeline -- host-to-device
+ * copies on one internal stream, the two kernels on `stream`, device-to-host copies on a second
+ * internal stream, chained by events -- so that both directions of the host link are busy at once.
+ *   workspace [scratch, device] at least nfad_host_step_workspace_bytes(dtype, n) bytes for full speed,
+ *             16-byte aligned; any size that holds one chunk of 2048 elements per slot works
+ *             (NFAD_E_SCRATCH below that).  Contents undefined afterwards.
+ * Host buffers should be page-locked (cudaHostAlloc / cudaHostRegister): pageable memory works but
+ * the copies then block the calling thread and do not overlap.  Host buffers must not overlap one
+ * another.  Completion is stream-ordered on `stream`: work enqueued on `stream` after the call, and a
+ * synchronisation on it, see every result in host memory.  flags = 0: the inputs are read in stream
+ * order too (the copies start when `stream` reaches the call).  flags = NFAD_HOST_INPUTS_READY: the
+ * caller guarantees that x_host and grad_out_host hold their final contents when the call is made
+ * and that no work pending on `stream` writes them; the input copies may then start at once, so
+ * that consecutive calls keep both directions of the link busy across the call boundary (a call
+ * whose workspace or chunk size differs from the previous one's first waits for that one to finish).
+ * Any other flag bit gives NFAD_E_LAYOUT.  State: two streams and a few events per
+ * device, created on the first call on that device (make that call outside a stream capture; the
+ * call itself cannot be captured into a graph) and kept until the process exits; enqueueing is
+ * serialised by a mutex.  After NFAD_E_CUDA, nfad_host_last_cuda_error() gives the cudaError_t.
+ */
+#define NFAD_HOST_INPUTS_READY 1
+NFAD_API int nfad_host_step(int kind, int dtype, const void* x_host, const void* grad_out_host, void* y_host, void* dfdx_host,
+                            void* grad_in_host, size_t n, void* workspace, size_t workspace_bytes, int flags,
+                            nfad_stream_t stream);
+NFAD_API size_t nfad_host_step_workspace_bytes(int dtype, size_t n);
+NFAD_API int nfad_host_last_cuda_error(void);
+
+/*
  * Traffic probe (a measurement aid with no counterpart in the paper): moves
  * n_words 32-bit words per tensor through the same streaming kernel as the
  * activation pass, with a read/write mix of 1:1 (o0 = a), 1:2 (o0 = a, o1 = ~a)

@@ -10,6 +10,6 @@ from .binding import (  # noqa: F401
     nfad_bias_act_backward, nfad_bias_act_backward_scratch_bytes, nfad_bias_act_forward,
     nfad_cmp_conv_backward, nfad_cmp_recompute_backward, nfad_cmp_recompute_backward_noalloc,
     nfad_cmp_recompute_scratch_bytes,
-    nfad_ew_op, nfad_probe_stream, nfad_saved_bytes_per_element, nfad_seq_backward, nfad_seq_forward,
+    nfad_ew_op, nfad_host_step, nfad_host_step_workspace_bytes, nfad_probe_stream, nfad_saved_bytes_per_element, nfad_seq_backward, nfad_seq_forward,
     nfad_status_string, nfad_version,
 )

@@ -32,6 +32,7 @@ EXPORTS = (
     "nfad_seq_forward", "nfad_seq_backward", "nfad_ew_op",
     "nfad_bias_act_forward", "nfad_bias_act_backward", "nfad_bias_act_backward_scratch_bytes",
     "nfad_act_forward_strict",
+    "nfad_host_step", "nfad_host_step_workspace_bytes", "nfad_host_last_cuda_error",
 )
 OPCODES = {"add": 0, "mul": 1, "scale": 2, "add_const": 3, "exp": 4, "log1p": 5, "tanh": 6, "erf": 7, "softplus": 8,
            "sigmoid": 9, "half_one_plus_tanh": 10, "half_one_plus_erf": 11, "out": 12}
@@ -86,6 +87,12 @@ def load() -> ctypes.CDLL:
         lib.nfad_bias_act_backward.restype = ci
         lib.nfad_bias_act_backward_scratch_bytes.argtypes = [ci, sz, sz]
         lib.nfad_bias_act_backward_scratch_bytes.restype = sz
+        lib.nfad_host_step.argtypes = [ci, ci, vp, vp, vp, vp, vp, sz, vp, sz, ci, vp]
+        lib.nfad_host_step.restype = ci
+        lib.nfad_host_step_workspace_bytes.argtypes = [ci, sz]
+        lib.nfad_host_step_workspace_bytes.restype = sz
+        lib.nfad_host_last_cuda_error.argtypes = []
+        lib.nfad_host_last_cuda_error.restype = ci
         lib.nfad_cmp_recompute_scratch_bytes.argtypes = [ci, ci, sz]
         lib.nfad_cmp_recompute_scratch_bytes.restype = sz
         lib.nfad_saved_bytes_per_element.argtypes = [ci, ci, ci]
@@ -267,6 +274,45 @@ def nfad_bias_act_backward(kind, grad_out: torch.Tensor, dfdx: torch.Tensor, gra
         _check(load().nfad_bias_act_backward(_kind(kind), _TORCH_TO_CODE[grad_out.dtype], pg, _tensor(dfdx, "dfdx", grad_out),
                                              _tensor(grad_in, "grad_in", grad_out), grad_bias.data_ptr(), sp, sb, rows, cols,
                                              _stream(grad_out)), "nfad_bias_act_backward")
+
+
+def _host_tensor(t: torch.Tensor, name: str, like: Optional[torch.Tensor] = None) -> int:
+    if not isinstance(t, torch.Tensor) or t.is_cuda:
+        raise TypeError(f"{name} must be a host tensor")
+    if t.dtype not in _TORCH_TO_CODE or not t.is_contiguous():
+        raise ValueError(f"{name} must be a contiguous float32 / bfloat16 / float16 tensor")
+    if like is not None and (t.dtype != like.dtype or t.numel() != like.numel()):
+        raise ValueError(f"{name} must match the first tensor's dtype and size")
+    return t.data_ptr()
+
+
+def nfad_host_step_workspace_bytes(dtype, n: int) -> int:
+    code = _TORCH_TO_CODE[dtype] if isinstance(dtype, torch.dtype) else DTYPES[dtype]
+    return int(load().nfad_host_step_workspace_bytes(code, n))
+
+
+HOST_INPUTS_READY = 1
+
+
+def nfad_host_step(kind, x_host: torch.Tensor, grad_out_host: torch.Tensor, y_host: torch.Tensor, dfdx_host,
+                   grad_in_host: torch.Tensor, workspace: torch.Tensor, inputs_ready: bool = False) -> None:
+    """Forward + backward for host (ideally pinned) tensors through the device `workspace` lives on; results are in
+    host memory once the current stream of that device has completed.  inputs_ready: the host inputs hold their
+    final contents now and nothing pending on the stream writes them (lets consecutive calls overlap)."""
+    px = _host_tensor(x_host, "x_host")
+    if not workspace.is_cuda or not workspace.is_contiguous():
+        raise TypeError("workspace must be a contiguous CUDA tensor")
+    lib = load()
+    with _on_device(workspace.device):
+        rc = lib.nfad_host_step(_kind(kind), _TORCH_TO_CODE[x_host.dtype], px, _host_tensor(grad_out_host, "grad_out_host", x_host),
+                                _host_tensor(y_host, "y_host", x_host),
+                                _host_tensor(dfdx_host, "dfdx_host", x_host) if dfdx_host is not None else None,
+                                _host_tensor(grad_in_host, "grad_in_host", x_host), x_host.numel(), workspace.data_ptr(),
+                                workspace.numel() * workspace.element_size(), HOST_INPUTS_READY if inputs_ready else 0,
+                                _stream(workspace))
+        if rc == 5:
+            raise RuntimeError(f"nfad_host_step: CUDA error {lib.nfad_host_last_cuda_error()}")
+        _check(rc, "nfad_host_step")
 
 
 def _ptr_array(tensors, name, like):

@@ -3,11 +3,11 @@
     python -m paper_2209_10778_b200.build          # rebuild if sources are newer
     python -m paper_2209_10778_b200.build --force
 
-Five translation units: the fp32-storage kernels are compiled with
+Six translation units: the fp32-storage kernels are compiled with
 floating-point contraction OFF (their compensated arithmetic depends on every
 fused multiply-add being written out), the 16-bit-storage kernels and the run-time
 sequences with it on, the bias-gradient kernels (explicitly rounded intrinsics only),
-and the extern "C" boundary.  No fast-math, no flush-to-zero, IEEE division:
+the extern "C" boundary, and the host-memory pipeline (no kernels of its own).  No fast-math, no flush-to-zero, IEEE division:
 subnormal inputs and results are part of the contract.
 """
 from __future__ import annotations
@@ -31,6 +31,7 @@ UNITS = [
     ("nfad_kernels_seq.cu", ["-fmad=true"]),
     ("nfad_kernels_bias.cu", ["-fmad=false"]),
     ("nfad_api.cu", ["-fmad=false"]),
+    ("nfad_host.cu", ["-fmad=false"]),
 ]
 
 
