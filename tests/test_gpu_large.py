@@ -19,10 +19,11 @@ DEV = "cuda"
 
 def _sample_indices(n: int, es: int) -> torch.Tensor:
     idx = [torch.arange(0, min(n, 20000)), torch.arange(max(0, n - 20000), n), torch.arange(0, n, 100003)]
-    per_tile = 4096 * 16 // es                       # elements per 256 x 4-packet tile
-    for k in (1, 2, 3, 1000, n // per_tile - 1, n // per_tile):
-        c = k * per_tile
-        idx.append(torch.arange(max(0, c - 40), min(n, c + 40)))
+    for packets in (4, 5):                           # elements per tile: 256 threads x 4 (or, 16-bit forward, 5) packets
+        per_tile = 256 * packets * 16 // es
+        for k in (1, 2, 3, 1000, n // per_tile - 1, n // per_tile):
+            c = k * per_tile
+            idx.append(torch.arange(max(0, c - 40), min(n, c + 40)))
     for byte_mark in (1 << 31, 1 << 32, 3 << 31):
         c = byte_mark // es
         if 40 < c < n - 40:
@@ -66,3 +67,38 @@ def test_bf16_beyond_two_to_the_thirty_one_elements_sampled():
 
 def test_fp16_quarter_billion_mix_sampled():
     _sampled_check("swish", "f16", 1 << 28, "mix")
+
+
+def test_bert_ffn_step_replayed_from_a_cuda_graph():
+    # the benchmark's launch configuration: the step's four launches (programmatic dependent launch between them)
+    # captured in a CUDA graph and replayed; every element of both kinds against the oracle
+    w = W.WORKLOADS["bert_base_ffn"]
+    x, g = W.workload_tensors(w, 0, DEV)
+    bufs = {k: [torch.empty_like(x) for _ in range(3)] for k in w.kinds}
+
+    def step():
+        for k in w.kinds:
+            y, d, gin = bufs[k]
+            nfad.nfad_act_forward(k, x, y, d)
+            nfad.nfad_act_backward(k, g, d, gin)
+
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        step()
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    for k in w.kinds:
+        for t in bufs[k]:
+            t.zero_()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        step()
+    graph.replay()
+    graph.replay()
+    torch.cuda.synchronize()
+    x_raw, g_raw = W.raw_numpy(x), W.raw_numpy(g)
+    for k in w.kinds:
+        y, d, gin = (W.raw_numpy(t) for t in bufs[k])
+        parity.check_forward_16(k, w.dtype, x_raw, y, d)
+        parity.check_backward(w.dtype, g_raw, d, gin)
