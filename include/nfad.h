@@ -236,6 +236,24 @@ NFAD_API int nfad_seq_forward(const nfad_seq_op* program, int n_ops, int dtype, 
                               void* const* dfdx, int m, size_t n, nfad_stream_t stream);
 
 /*
+ * Two executors run a sequence.  The COMPILED one turns the program into straight-line device code
+ * over the same dual primitives, compiles it for the device at hand with NVRTC on first use (about a
+ * second per new (program, dtype, m); cached afterwards) and launches it as one kernel with every
+ * dual number in hardware registers, like the dedicated activation kernels.  The INTERPRETER runs any
+ * program at once with its registers in local memory and is several times slower.  Mode 0 (the
+ * default): compiled when NVRTC, the driver library and this library's headers (the csrc directory
+ * beside the library, or NFAD_JIT_INCLUDE) are available, otherwise interpreted; 1: always
+ * interpreted; 2: compiled or fail (NFAD_E_CUDA with cudaErrorNotSupported or the compiler's error,
+ * whose text nfad_seq_compile_log() returns).  The two executors run the same primitives, but the
+ * compiler may contract across instruction boundaries: results can differ in the last bits.
+ * nfad_seq_last_executor(): 1 = interpreter, 2 = compiled, for the calling thread's last sequence.
+ * The first compiled call of a program must not be made inside a stream capture.
+ */
+NFAD_API int nfad_seq_set_executor(int mode);
+NFAD_API int nfad_seq_last_executor(void);
+NFAD_API const char* nfad_seq_compile_log(void);
+
+/*
  * Backward of a sequence with m results (Section II-E; for a binary merge "the post-process
  * will merge (accumulate) FAD results", Section IV): grad_in[i] = sum_k grad_out[k][i] * dfdx[k][i],
  * accumulated in fp32 in the order k = 0..m-1 with fused multiply-adds and rounded once.

@@ -33,6 +33,7 @@ EXPORTS = (
     "nfad_bias_act_forward", "nfad_bias_act_backward", "nfad_bias_act_backward_scratch_bytes",
     "nfad_act_forward_strict",
     "nfad_host_step", "nfad_host_step_workspace_bytes", "nfad_host_last_cuda_error",
+    "nfad_seq_set_executor", "nfad_seq_last_executor", "nfad_seq_compile_log",
 )
 OPCODES = {"add": 0, "mul": 1, "scale": 2, "add_const": 3, "exp": 4, "log1p": 5, "tanh": 6, "erf": 7, "softplus": 8,
            "sigmoid": 9, "half_one_plus_tanh": 10, "half_one_plus_erf": 11, "out": 12}
@@ -87,6 +88,12 @@ def load() -> ctypes.CDLL:
         lib.nfad_bias_act_backward.restype = ci
         lib.nfad_bias_act_backward_scratch_bytes.argtypes = [ci, sz, sz]
         lib.nfad_bias_act_backward_scratch_bytes.restype = sz
+        lib.nfad_seq_set_executor.argtypes = [ci]
+        lib.nfad_seq_set_executor.restype = ci
+        lib.nfad_seq_last_executor.argtypes = []
+        lib.nfad_seq_last_executor.restype = ci
+        lib.nfad_seq_compile_log.argtypes = []
+        lib.nfad_seq_compile_log.restype = ctypes.c_char_p
         lib.nfad_host_step.argtypes = [ci, ci, vp, vp, vp, vp, vp, sz, vp, sz, ci, vp]
         lib.nfad_host_step.restype = ci
         lib.nfad_host_step_workspace_bytes.argtypes = [ci, sz]
@@ -338,6 +345,21 @@ def nfad_seq_forward(program, x: torch.Tensor, ys, dfdxs) -> None:
     with _on_device(x.device):
         _check(load().nfad_seq_forward(ops, len(program), _TORCH_TO_CODE[x.dtype], px, _ptr_array(ys, "y", x),
                                        _ptr_array(dfdxs, "dfdx", x), len(ys), x.numel(), _stream(x)), "nfad_seq_forward")
+
+
+SEQ_EXECUTORS = {"auto": 0, "interpreter": 1, "compiled": 2}
+
+
+def nfad_seq_set_executor(mode) -> None:
+    _check(load().nfad_seq_set_executor(SEQ_EXECUTORS[mode] if isinstance(mode, str) else int(mode)), "nfad_seq_set_executor")
+
+
+def nfad_seq_last_executor() -> str:
+    return {0: "none", 1: "interpreter", 2: "compiled"}[load().nfad_seq_last_executor()]
+
+
+def nfad_seq_compile_log() -> str:
+    return load().nfad_seq_compile_log().decode(errors="replace")
 
 
 def nfad_seq_backward(grad_outs, dfdxs, grad_in: torch.Tensor) -> None:

@@ -3,11 +3,11 @@
     python -m paper_2209_10778_b200.build          # rebuild if sources are newer
     python -m paper_2209_10778_b200.build --force
 
-Six translation units: the fp32-storage kernels are compiled with
+Seven translation units: the fp32-storage kernels are compiled with
 floating-point contraction OFF (their compensated arithmetic depends on every
 fused multiply-add being written out), the 16-bit-storage kernels and the run-time
 sequences with it on, the bias-gradient kernels (explicitly rounded intrinsics only),
-the extern "C" boundary, and the host-memory pipeline (no kernels of its own).  No fast-math, no flush-to-zero, IEEE division:
+the extern "C" boundary, the host-memory pipeline and the run-time compiler of FAD sequences (no kernels of their own).  No fast-math, no flush-to-zero, IEEE division:
 subnormal inputs and results are part of the contract.
 """
 from __future__ import annotations
@@ -32,6 +32,7 @@ UNITS = [
     ("nfad_kernels_bias.cu", ["-fmad=false"]),
     ("nfad_api.cu", ["-fmad=false"]),
     ("nfad_host.cu", ["-fmad=false"]),
+    ("nfad_jit.cu", ["-fmad=false"]),
 ]
 
 
@@ -77,7 +78,7 @@ def build_library(force: bool = False, verbose: bool = False) -> str:
         if p.returncode != 0:
             raise RuntimeError("nvcc failed:\n" + " ".join(cmd) + "\n" + (out or ""))
     # the extern "C" entry points are the only exported symbols
-    link = [nvcc, *ARCH, "-shared", "-o", LIB, *objs, "-Xcompiler", "-fPIC", "-cudart", "static"]
+    link = [nvcc, *ARCH, "-shared", "-o", LIB, *objs, "-Xcompiler", "-fPIC", "-cudart", "static", "-ldl"]
     r = subprocess.run(link, capture_output=True, text=True)
     if r.returncode != 0:
         raise RuntimeError("link failed:\n" + r.stdout + r.stderr)

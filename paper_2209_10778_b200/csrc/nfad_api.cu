@@ -326,7 +326,7 @@ int nfad_seq_forward(const nfad_seq_op* program, int n_ops, int dtype, const voi
     if (dtype < 0 || dtype > 2) return NFAD_E_DTYPE;
     if (!program || !y || !dfdx) return NFAD_E_NULL;
     if (n_ops < 1 || n_ops > nfad::kSeqMaxOpsHost || m < 1 || m > 4) return NFAD_E_PROGRAM;
-    nfad::SeqProgramHost p;
+    nfad::SeqProgramHost p = {};
     p.n_ops = n_ops;
     constexpr int kRegs = 12;
     bool written[kRegs] = {true};
@@ -359,6 +359,17 @@ int nfad_seq_forward(const nfad_seq_op* program, int n_ops, int dtype, const voi
     return NFAD_OK;
 }
 
+int nfad_seq_set_executor(int mode)
+{
+    if (mode < 0 || mode > 2) return NFAD_E_LAYOUT;
+    nfad::seq_set_executor_mode(mode);
+    return NFAD_OK;
+}
+
+int nfad_seq_last_executor(void) { return nfad::seq_last_executor(); }
+
+const char* nfad_seq_compile_log(void) { return nfad::seq_jit_log(); }
+
 int nfad_seq_backward(int dtype, const void* const* grad_out, const void* const* dfdx, int m, void* grad_in, size_t n,
                       nfad_stream_t stream)
 {
@@ -371,6 +382,10 @@ int nfad_seq_backward(int dtype, const void* const* grad_out, const void* const*
     int rc = check(0, dtype, in, 2 * m, out, 1, n);
     if (rc) return rc;
     if (n == 0) return NFAD_OK;
+    if (m == 1) {                                   // one result: exactly the multiplication of nfad_act_backward
+        const void* in1[2] = {grad_out[0], dfdx[0]};
+        return run(nfad::kOpBackward, 0, dtype, in1, out, n, stream);
+    }
     cudaError_t e = nfad::launch_seq_backward(dtype, grad_out, dfdx, m, grad_in, n, static_cast<cudaStream_t>(stream));
     if (e != cudaSuccess) { g_last_cuda_error = static_cast<int>(e); return NFAD_E_CUDA; }
     return NFAD_OK;

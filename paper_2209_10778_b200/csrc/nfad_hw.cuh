@@ -4,7 +4,9 @@
 // fixed by the source text alone.
 #pragma once
 
+#ifndef __CUDACC_RTC__
 #include <cuda_runtime.h>
+#endif
 
 #define NFAD_DEV __device__ __forceinline__
 

@@ -35,6 +35,14 @@ struct SeqProgramHost { int n_ops; int op[kSeqMaxOpsHost], a[kSeqMaxOpsHost], b[
 
 cudaError_t launch_seq_forward(const SeqProgramHost& p, int dtype, const void* x, void* const* y, void* const* d, int m, size_t n,
                                cudaStream_t st);
+// The same sequence compiled at run time into one kernel (nfad_jit.cu).  cudaErrorNotSupported: not available here.
+cudaError_t launch_seq_forward_compiled(const SeqProgramHost& p, int dtype, const void* x, void* const* y, void* const* d, int m,
+                                        size_t n, cudaStream_t st);
+int seq_executor_mode();                 // 0 automatic, 1 interpreter only, 2 compiled only
+void seq_set_executor_mode(int mode);
+int seq_last_executor();                 // of the calling thread: 0 none yet, 1 interpreter, 2 compiled
+void seq_note_executor(int which);
+const char* seq_jit_log();
 cudaError_t launch_seq_backward(int dtype, const void* const* g, const void* const* d, int m, void* gin, size_t n, cudaStream_t st);
 cudaError_t launch_ew(int op, int backward, float c, int dtype, const void* const* in, void* const* out, size_t n, cudaStream_t st);
 

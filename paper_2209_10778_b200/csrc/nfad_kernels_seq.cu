@@ -94,6 +94,16 @@ cudaError_t ew_t(int op, int backward, float c, const void* const* in, void* con
 cudaError_t launch_seq_forward(const SeqProgramHost& p, int dtype, const void* x, void* const* y, void* const* d, int m, size_t n,
                                cudaStream_t st)
 {
+    const int mode = seq_executor_mode();
+    if (mode != 1) {
+        cudaError_t e = launch_seq_forward_compiled(p, dtype, x, y, d, m, n, st);
+        if (e == cudaSuccess) {
+            seq_note_executor(2);
+            return e;
+        }
+        if (mode == 2 || e != cudaErrorNotSupported) return e;
+    }
+    seq_note_executor(1);
     SeqProgram prog;
     prog.n_ops = p.n_ops;
     for (int i = 0; i < p.n_ops; ++i) prog.ops[i] = SeqOp{p.op[i], p.a[i], p.b[i], p.dst[i], p.c[i]};

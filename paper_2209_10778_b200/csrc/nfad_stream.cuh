@@ -14,10 +14,10 @@
 // scalar paths agree bit for bit.
 #pragma once
 
-#include <cuda_bf16.h>
-#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
+
+#include "nfad_storage.cuh"
 
 namespace nfad {
 
@@ -26,106 +26,6 @@ constexpr int kBlock = 256;
 #define NFAD_UNROLL 4
 #endif
 constexpr int kDefaultUnroll = NFAD_UNROLL;
-// Resident CTAs per SM the compiler must leave room for (a register cap).  The 16-bit kernels
-// are issue-bound with short dependency chains through MUFU: 5 CTAs (40 warps, <= 48 registers)
-// measured 3-5 % faster than the 4 the compiler picks by itself (7 or more spill and lose 30 %); the fp32 kernels need their
-// ~48 registers (a tighter cap spills).
-#ifndef NFAD_PDL
-#define NFAD_PDL 1
-#endif
-#ifndef NFAD_MIN_BLOCKS_16
-#define NFAD_MIN_BLOCKS_16 5
-#endif
-#ifndef NFAD_MIN_BLOCKS_32
-#define NFAD_MIN_BLOCKS_32 5
-#endif
-
-// ---------------------------------------------------------------- storage types
-
-struct StoreF32 {
-    using elem = float;
-    static constexpr int kVec = 4;             // elements per 16-byte packet
-    static constexpr int kMinBlocks = NFAD_MIN_BLOCKS_32;
-    static __device__ __forceinline__ void unpack(const uint4& p, float (&v)[4])
-    {
-        v[0] = __uint_as_float(p.x); v[1] = __uint_as_float(p.y);
-        v[2] = __uint_as_float(p.z); v[3] = __uint_as_float(p.w);
-    }
-    static __device__ __forceinline__ uint4 pack(const float (&v)[4])
-    {
-        return make_uint4(__float_as_uint(v[0]), __float_as_uint(v[1]), __float_as_uint(v[2]), __float_as_uint(v[3]));
-    }
-    static __device__ __forceinline__ float load1(const elem* p) { return *p; }
-    static __device__ __forceinline__ void store1(elem* p, float v) { *p = v; }
-};
-
-struct StoreBF16 {
-    using elem = __nv_bfloat16;
-    static constexpr int kVec = 8;
-    static constexpr int kMinBlocks = NFAD_MIN_BLOCKS_16;
-    // a bf16 is the upper half of an fp32: widening is a shift or a mask
-    static __device__ __forceinline__ void unpack(const uint4& p, float (&v)[8])
-    {
-        const uint32_t w[4] = {p.x, p.y, p.z, p.w};
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            v[2 * i] = __uint_as_float(w[i] << 16);
-            v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
-        }
-    }
-    static __device__ __forceinline__ uint32_t pack2(float lo, float hi)
-    {
-        __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);   // cvt.rn.bf16x2.f32: round to nearest even
-        return *reinterpret_cast<uint32_t*>(&h);
-    }
-    static __device__ __forceinline__ uint4 pack(const float (&v)[8])
-    {
-        return make_uint4(pack2(v[0], v[1]), pack2(v[2], v[3]), pack2(v[4], v[5]), pack2(v[6], v[7]));
-    }
-    static __device__ __forceinline__ float load1(const elem* p) { return __bfloat162float(*p); }
-    static __device__ __forceinline__ void store1(elem* p, float v) { *p = __float2bfloat16_rn(v); }
-};
-
-struct StoreF16 {
-    using elem = __half;
-    static constexpr int kVec = 8;
-    static constexpr int kMinBlocks = NFAD_MIN_BLOCKS_16;
-    static __device__ __forceinline__ void unpack(const uint4& p, float (&v)[8])
-    {
-        const uint32_t w[4] = {p.x, p.y, p.z, p.w};
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            float2 f = __half22float2(*reinterpret_cast<const __half2*>(&w[i]));
-            v[2 * i] = f.x;
-            v[2 * i + 1] = f.y;
-        }
-    }
-    static __device__ __forceinline__ uint32_t pack2(float lo, float hi)
-    {
-        __half2 h = __floats2half2_rn(lo, hi);              // cvt.rn.f16x2.f32
-        return *reinterpret_cast<uint32_t*>(&h);
-    }
-    static __device__ __forceinline__ uint4 pack(const float (&v)[8])
-    {
-        return make_uint4(pack2(v[0], v[1]), pack2(v[2], v[3]), pack2(v[4], v[5]), pack2(v[6], v[7]));
-    }
-    static __device__ __forceinline__ float load1(const elem* p) { return __half2float(*p); }
-    static __device__ __forceinline__ void store1(elem* p, float v) { *p = __float2half_rn(v); }
-};
-
-// ---------------------------------------------------------------- memory access with cache hints
-
-// Inputs are read once: streaming (evict-first) loads.
-__device__ __forceinline__ uint4 load_packet(const uint4* p) { return __ldcs(p); }
-
-// Output slot `keep`: true for a tensor the next kernel reads at once (y, grad_in),
-// false for one that is read much later or never by this stream (the saved f').
-template <bool kKeep> __device__ __forceinline__ void store_packet(uint4* p, const uint4& v)
-{
-    if (kKeep) *p = v;
-    else __stcs(p, v);
-}
-
 // ---------------------------------------------------------------- kernel
 
 template <int NIN, int NOUT> struct StreamArgs {

@@ -196,6 +196,14 @@ def run_opbyop(n: int, dtype: str, kinds, reps: int = 5, dev="cuda"):
             nfad.nfad_seq_forward(prog.ops, x, [y], [d])
             nfad.nfad_seq_backward([g], [d], gin)
 
+        def compiled_seq():
+            nfad.nfad_seq_set_executor("compiled")
+            fused_seq()
+
+        def interpreted_seq():
+            nfad.nfad_seq_set_executor("interpreter")
+            fused_seq()
+
         ex = sequence.OpByOp(prog)
         kept = {}
 
@@ -204,7 +212,9 @@ def run_opbyop(n: int, dtype: str, kinds, reps: int = 5, dev="cuda"):
             kept["bytes"] = ex.saved_bytes()
             ex.backward([g])
 
-        rows = [("nested (dedicated kernels)", nested, n * es), ("nested (run-time sequence)", fused_seq, n * es),
+        rows = [("nested (dedicated kernels)", nested, n * es),
+                ("nested (run-time sequence, compiled)", compiled_seq, n * es),
+                ("nested (run-time sequence, interpreted)", interpreted_seq, n * es),
                 ("operator by operator", op_by_op, None)]
         for name, fn, saved in rows:
             ms = timed(fn)
@@ -213,6 +223,7 @@ def run_opbyop(n: int, dtype: str, kinds, reps: int = 5, dev="cuda"):
                         "kept_tensors": (saved if saved is not None else kept["bytes"]) / (n * es),
                         "launches": 2 if saved is not None else None})
             torch.cuda.empty_cache()
+    nfad.nfad_seq_set_executor("auto")
     return out
 
 

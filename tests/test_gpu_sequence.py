@@ -50,14 +50,27 @@ def _close(dtype, got_t, want64, x64):
     return ok
 
 
+@pytest.fixture(params=["interpreter", "compiled"])
+def executor(request):
+    """Runs a test under each of the two executors of a sequence; the compiled one must really be the one that ran."""
+    nfad.nfad_seq_set_executor(request.param)
+    yield request.param
+    nfad.nfad_seq_set_executor("auto")
+
+
 @pytest.mark.parametrize("name", list(PROGRAMS))
 @pytest.mark.parametrize("dtype", ["f32", "bf16", "f16"])
-def test_fused_executor_against_the_sequence_oracle(name, dtype):
+def test_fused_executor_against_the_sequence_oracle(name, dtype, executor):
     prog = PROGRAMS[name]()
     n = 70001
     x = (W.normal(n, "f32", 5, 2.0, DEV).clamp_(-7, 7)).to(W.TORCH_DTYPES[dtype])
-    ys, ds = sequence.run_fused(prog, x)
+    try:
+        ys, ds = sequence.run_fused(prog, x)
+    except Exception:
+        print(nfad.nfad_seq_compile_log())
+        raise
     torch.cuda.synchronize()
+    assert nfad.nfad_seq_last_executor() == executor
     x64 = oracle.widen(dtype, W.raw_numpy(x))
     y, d = oracle.seq_forward(prog.ops, x64, prog.n_out)
     for k in range(prog.n_out):
@@ -65,8 +78,27 @@ def test_fused_executor_against_the_sequence_oracle(name, dtype):
         assert _close(dtype, ds[k], d[k], x64).all(), (name, dtype, "derivative", k)
 
 
+def test_automatic_mode_compiles_and_caches():
+    import time
+    nfad.nfad_seq_set_executor("auto")
+    p = sequence.FadProgram()
+    p.output(p.unary("tanh", p.scale(0.37, p.x())))          # a program no other test uses: first call compiles
+    x = W.normal(1 << 20, "bf16", 9, 1.0, DEV)
+    t0 = time.perf_counter()
+    sequence.run_fused(p, x)
+    torch.cuda.synchronize()
+    first = time.perf_counter() - t0
+    assert nfad.nfad_seq_last_executor() == "compiled", nfad.nfad_seq_compile_log()
+    t0 = time.perf_counter()
+    for _ in range(10):
+        sequence.run_fused(p, x)
+    torch.cuda.synchronize()
+    later = (time.perf_counter() - t0) / 10
+    assert later < first / 20, (first, later)                # cached: no recompilation
+
+
 @pytest.mark.parametrize("dtype", ["f32", "bf16", "f16"])
-def test_fused_executor_edges_and_unaligned(dtype):
+def test_fused_executor_edges_and_unaligned(dtype, executor):
     prog = sequence.swish_program()
     td = W.TORCH_DTYPES[dtype]
     for n in (1, 7, 8, 9, 255, 257, 4099):
