@@ -346,14 +346,13 @@ NFAD_API size_t nfad_bias_act_backward_scratch_bytes(int dtype, size_t rows, siz
  * Any other flag bit gives NFAD_E_LAYOUT.  State: two streams and a few events per
  * device, created on the first call on that device (make that call outside a stream capture; the
  * call itself cannot be captured into a graph) and kept until the process exits; enqueueing is
- * serialised by a mutex.  After NFAD_E_CUDA, nfad_host_last_cuda_error() gives the cudaError_t.
+ * serialised by a mutex.
  */
 #define NFAD_HOST_INPUTS_READY 1
 NFAD_API int nfad_host_step(int kind, int dtype, const void* x_host, const void* grad_out_host, void* y_host, void* dfdx_host,
                             void* grad_in_host, size_t n, void* workspace, size_t workspace_bytes, int flags,
                             nfad_stream_t stream);
 NFAD_API size_t nfad_host_step_workspace_bytes(int dtype, size_t n);
-NFAD_API int nfad_host_last_cuda_error(void);
 
 /*
  * Traffic probe (a measurement aid with no counterpart in the paper): moves

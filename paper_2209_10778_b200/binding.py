@@ -32,7 +32,7 @@ EXPORTS = (
     "nfad_seq_forward", "nfad_seq_backward", "nfad_ew_op",
     "nfad_bias_act_forward", "nfad_bias_act_backward", "nfad_bias_act_backward_scratch_bytes",
     "nfad_act_forward_strict",
-    "nfad_host_step", "nfad_host_step_workspace_bytes", "nfad_host_last_cuda_error",
+    "nfad_host_step", "nfad_host_step_workspace_bytes",
     "nfad_seq_set_executor", "nfad_seq_last_executor", "nfad_seq_compile_log",
 )
 OPCODES = {"add": 0, "mul": 1, "scale": 2, "add_const": 3, "exp": 4, "log1p": 5, "tanh": 6, "erf": 7, "softplus": 8,
@@ -98,8 +98,6 @@ def load() -> ctypes.CDLL:
         lib.nfad_host_step.restype = ci
         lib.nfad_host_step_workspace_bytes.argtypes = [ci, sz]
         lib.nfad_host_step_workspace_bytes.restype = sz
-        lib.nfad_host_last_cuda_error.argtypes = []
-        lib.nfad_host_last_cuda_error.restype = ci
         lib.nfad_cmp_recompute_scratch_bytes.argtypes = [ci, ci, sz]
         lib.nfad_cmp_recompute_scratch_bytes.restype = sz
         lib.nfad_saved_bytes_per_element.argtypes = [ci, ci, ci]
@@ -317,8 +315,6 @@ def nfad_host_step(kind, x_host: torch.Tensor, grad_out_host: torch.Tensor, y_ho
                                 _host_tensor(grad_in_host, "grad_in_host", x_host), x_host.numel(), workspace.data_ptr(),
                                 workspace.numel() * workspace.element_size(), HOST_INPUTS_READY if inputs_ready else 0,
                                 _stream(workspace))
-        if rc == 5:
-            raise RuntimeError(f"nfad_host_step: CUDA error {lib.nfad_host_last_cuda_error()}")
         _check(rc, "nfad_host_step")
 
 

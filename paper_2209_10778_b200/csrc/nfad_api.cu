@@ -106,6 +106,10 @@ cudaError_t noalloc_scratch(void** out)
 
 }  // namespace
 
+namespace nfad {
+void note_cuda_error(cudaError_t e) { g_last_cuda_error = static_cast<int>(e); }
+}  // namespace nfad
+
 extern "C" {
 
 int nfad_act_forward(int kind, int dtype, const void* x, void* y, void* dfdx, size_t n, nfad_stream_t stream)

@@ -16,6 +16,7 @@
 #include <mutex>
 
 #include "../../include/nfad.h"
+#include "nfad_internal.h"
 
 namespace {
 
@@ -80,8 +81,6 @@ size_t chunk_elements(int dtype, size_t n, size_t bytes)
     return c;
 }
 
-thread_local int g_last_host_cuda_error = 0;
-
 }  // namespace
 
 extern "C" {
@@ -95,8 +94,6 @@ size_t nfad_host_step_workspace_bytes(int dtype, size_t n)
     if (c > n_up) c = n_up;
     return size_t(kSlots) * 5 * c * es;
 }
-
-int nfad_host_last_cuda_error(void) { return g_last_host_cuda_error; }
 
 int nfad_host_step(int kind, int dtype, const void* x_host, const void* grad_out_host, void* y_host, void* dfdx_host,
                    void* grad_in_host, size_t n, void* workspace, size_t workspace_bytes, int flags, nfad_stream_t stream)
@@ -116,7 +113,7 @@ int nfad_host_step(int kind, int dtype, const void* x_host, const void* grad_out
     cudaError_t e = device_state(&s);
     cudaStream_t compute = static_cast<cudaStream_t>(stream);
     auto fail = [&](cudaError_t err) {
-        g_last_host_cuda_error = static_cast<int>(err);
+        nfad::note_cuda_error(err);
         return NFAD_E_CUDA;
     };
     if (e != cudaSuccess) return fail(e);
@@ -160,10 +157,7 @@ int nfad_host_step(int kind, int dtype, const void* x_host, const void* grad_out
         if ((e = cudaStreamWaitEvent(compute, s->in[slot], 0)) != cudaSuccess) return fail(e);
         int rc = nfad_act_forward(kind, dtype, dx, dy, dd, m, stream);
         if (rc == NFAD_OK) rc = nfad_act_backward(kind, dtype, dg, dd, dgin, m, stream);
-        if (rc != NFAD_OK) {
-            if (rc == NFAD_E_CUDA) g_last_host_cuda_error = nfad_last_cuda_error();
-            return rc;
-        }
+        if (rc != NFAD_OK) return rc;
         if ((e = cudaEventRecord(s->done[slot], compute)) != cudaSuccess) return fail(e);
 
         // stage 3: results out

@@ -46,6 +46,9 @@ const char* seq_jit_log();
 cudaError_t launch_seq_backward(int dtype, const void* const* g, const void* const* d, int m, void* gin, size_t n, cudaStream_t st);
 cudaError_t launch_ew(int op, int backward, float c, int dtype, const void* const* in, void* const* out, size_t n, cudaStream_t st);
 
+// Records the cudaError_t behind an NFAD_E_CUDA of the calling thread (what nfad_last_cuda_error() returns).
+void note_cuda_error(cudaError_t e);
+
 // The pass fused with its producer's bias (nfad_bias.cuh).  x, y, d, g, gin: [rows, cols] row-major; bias: [cols].
 cudaError_t launch_bias_forward_f32(int kind, const void* x, const void* bias, void* y, void* d, size_t rows, size_t cols,
                                     cudaStream_t st);
