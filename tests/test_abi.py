@@ -78,3 +78,38 @@ def test_binding_refuses_cpu_tensors():
     x = torch.zeros(8)
     with pytest.raises(TypeError):
         binding.nfad_act_forward("swish", x, x.clone(), x.clone())
+
+
+def test_newer_entry_points_validate_without_a_device(lib):
+    fake, other = ctypes.c_void_p(0x10000), ctypes.c_void_p(0x90000)
+    # bias-fused pass: shape limits and pointers are checked before any CUDA call
+    assert lib.nfad_bias_act_forward(0, 0, fake, other, fake, ctypes.c_void_p(0x50000), 4, 1 << 31, None) == 9
+    assert lib.nfad_bias_act_forward(5, 0, fake, other, fake, fake, 4, 8, None) == 1
+    assert lib.nfad_bias_act_forward(0, 0, fake, None, ctypes.c_void_p(0x20000), ctypes.c_void_p(0x30000), 4, 8, None) == 3
+    assert lib.nfad_bias_act_forward(0, 0, None, None, None, None, 0, 8, None) == 0
+    assert lib.nfad_bias_act_backward(0, 4, fake, fake, fake, None, None, 0, 4, 8, None) == 2
+    # strict forward is fp32 only
+    assert lib.nfad_act_forward_strict(0, 1, fake, other, ctypes.c_void_p(0x50000), 8, None) == 2
+    assert lib.nfad_act_forward_strict(0, 0, None, None, None, 0, None) == 0
+    # host pipeline
+    assert lib.nfad_host_step(0, 0, fake, fake, fake, None, fake, 8, None, 0, 0, None) == 3
+    assert lib.nfad_host_step(0, 0, fake, fake, fake, None, fake, 8, fake, 1 << 20, 4, None) == 8
+    assert lib.nfad_host_step_workspace_bytes(1, 1 << 24) == 4 * 5 * (8 << 20)
+    assert lib.nfad_host_step_workspace_bytes(0, 1000) == 4 * 5 * 2048 * 4
+    assert lib.nfad_host_step_workspace_bytes(7, 1000) == 0
+    # executors of a run-time sequence
+    assert lib.nfad_seq_set_executor(3) == 8 and lib.nfad_seq_set_executor(-1) == 8
+    assert lib.nfad_seq_set_executor(1) == 0 and lib.nfad_seq_set_executor(0) == 0
+    assert lib.nfad_seq_last_executor() in (0, 1, 2)
+    # one-sided probes
+    assert lib.nfad_probe_stream(1, 0, ctypes.c_void_p(0x10004), None, other, None, 1024, None) == 6
+    assert lib.nfad_probe_stream(0, 1, None, None, None, None, 1024, None) == 3
+
+
+def test_binding_refuses_wrong_placements():
+    import torch
+    x = torch.zeros(8)
+    with pytest.raises(TypeError):
+        binding.nfad_bias_act_forward("swish", x, x.clone(), x.clone(), x.clone())
+    with pytest.raises(TypeError):
+        binding.nfad_act_forward_strict("swish", x, x.clone(), x.clone())
