@@ -365,6 +365,7 @@ def main(argv=None):
     ap.add_argument("--ops", default="forward,backward")
     ap.add_argument("--reps", type=int, default=20)
     ap.add_argument("--max-log2", type=int, default=30)
+    ap.add_argument("--repeats", type=int, default=10, help="bursts per case (1 under a profiler: the burst is then `reps` launches)")
     args = ap.parse_args(argv)
     if not torch.cuda.is_available():
         raise RuntimeError("needs a CUDA device")
@@ -427,7 +428,7 @@ def _run_config(args):
         for dtype in dtypes:
             for kind in kinds:
                 for op in ops:
-                    print(json.dumps(time_case(kind, dtype, op, args.n, args.reps)), flush=True)
+                    print(json.dumps(time_case(kind, dtype, op, args.n, args.reps, cols=args.cols, repeats=args.repeats)), flush=True)
                     torch.cuda.empty_cache()
 
 
