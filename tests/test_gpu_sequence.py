@@ -54,6 +54,17 @@ def _close(dtype, got_t, want64, x64):
 def executor(request):
     """Runs a test under each of the two executors of a sequence; the compiled one must really be the one that ran."""
     nfad.nfad_seq_set_executor(request.param)
+    if request.param == "compiled":
+        # a machine without the run-time compiler's libraries cannot run these cases (it would use the interpreter)
+        try:
+            x = torch.zeros(64, device=DEV)
+            sequence.run_fused(sequence.swish_program(), x)
+        except nfad.NfadError:
+            log = nfad.nfad_seq_compile_log()
+            nfad.nfad_seq_set_executor("auto")
+            if "not found" in log:
+                pytest.skip(f"run-time compiler unavailable here: {log}")
+            raise AssertionError(f"the compiled executor failed: {log}")
     yield request.param
     nfad.nfad_seq_set_executor("auto")
 
