@@ -488,6 +488,17 @@ template <class K> NFAD_DEV ActOut evaluate(K, Fast, float x)
 
 template <class K, class P> NFAD_DEV ActOut evaluate(float x) { return evaluate(K{}, P{}, x); }
 
+// x -> f(x) alone (a pass that will not be differentiated).  Same chain, same bits as evaluate().y; under the
+// Fast policy only the side that needs it is clamped: +inf goes through as it is (every gate is exactly 1
+// there, so f = x), -inf becomes the most negative float so that 0 * x gives -0.
+template <class K> NFAD_DEV float evaluate_value(K, Full, float x) { return evaluate(K{}, Full{}, x).y; }
+template <class K> NFAD_DEV float evaluate_value(K, Fast, float x)
+{
+    if (Saturation<K>::kFastClamp) return evaluate(K{}, Fast{}, x).y;
+    const float xf = hw::max_nan(x, -3.40282347e+38f);
+    return dual_value(dual_mul(Seed{xf}, gate<Fast>(K{}, Seed{xf})));
+}
+
 // x -> h(x) alone (what a recomputation pass re-materialises).
 template <class K, class P> NFAD_DEV float evaluate_gate(float x)
 {

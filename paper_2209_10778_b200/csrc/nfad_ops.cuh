@@ -36,7 +36,7 @@ template <class K, class P> struct ForwardInferOp {
     static __device__ __forceinline__ constexpr bool keep(int) { return true; }
     static __device__ __forceinline__ void apply(const float (&in)[1], float (&out)[1])
     {
-        out[0] = evaluate<K, P>(in[0]).y;
+        out[0] = evaluate_value(K{}, P{}, in[0]);
     }
 };
 
