@@ -12,11 +12,14 @@ namespace nfad {
 template <class P> struct IsFast { static constexpr bool value = false; };
 template <> struct IsFast<Fast> { static constexpr bool value = true; };
 
+#ifndef NFAD_FWD16_UNROLL
+#define NFAD_FWD16_UNROLL 5
+#endif
 template <class K, class P> struct ForwardTrainOp {
     static constexpr bool kPacketFixup = false;
     static constexpr int kMinBlocks = 0;
     // 16-bit storage: 5 packets per thread measured 1-4 % faster than 4 (3 and 6 are slower)
-    static constexpr int kUnroll = IsFast<P>::value ? 5 : 0;
+    static constexpr int kUnroll = IsFast<P>::value ? NFAD_FWD16_UNROLL : 0;
     static constexpr int kIn = 1, kOut = 2;
     static __device__ __forceinline__ constexpr bool keep(int k) { return k == 0; }   // y is consumed next; f' much later
     static __device__ __forceinline__ void apply(const float (&in)[1], float (&out)[2])
@@ -54,11 +57,17 @@ static __device__ __noinline__ float bf16_tiny_product(float g, float d)
     return (float)pd;
 }
 
+#ifndef NFAD_BWD_MIN_BLOCKS
+#define NFAD_BWD_MIN_BLOCKS 4
+#endif
+#ifndef NFAD_BWD_UNROLL
+#define NFAD_BWD_UNROLL 0
+#endif
 template <bool kBf16> struct BackwardOp {
     static constexpr int kIn = 2, kOut = 1;
     static constexpr bool kPacketFixup = kBf16;
-    static constexpr int kMinBlocks = 4;        // measured: 7 % faster than 5 for this load-and-multiply kernel
-    static constexpr int kUnroll = 0;
+    static constexpr int kMinBlocks = NFAD_BWD_MIN_BLOCKS;   // measured: 4 is 7 % faster than 5 for this load-and-multiply kernel
+    static constexpr int kUnroll = NFAD_BWD_UNROLL;
     static __device__ __forceinline__ constexpr bool keep(int) { return true; }
     static __device__ __forceinline__ void apply(const float (&in)[2], float (&out)[1]) { out[0] = in[0] * in[1]; }
     // scalar path (edges): the same result, element by element
