@@ -113,3 +113,26 @@ def test_binding_refuses_wrong_placements():
         binding.nfad_bias_act_forward("swish", x, x.clone(), x.clone(), x.clone())
     with pytest.raises(TypeError):
         binding.nfad_act_forward_strict("swish", x, x.clone(), x.clone())
+
+
+def test_sequence_programs_are_validated_without_a_device(lib):
+    Op = binding.SeqOp
+    fake = ctypes.c_void_p(0x10000)
+    outs = (ctypes.c_void_p * 1)(0x20000)
+    ds = (ctypes.c_void_p * 1)(0x30000)
+
+    def run(ops, m=1, n=0):
+        arr = (Op * len(ops))(*[Op(*o) for o in ops])
+        return lib.nfad_seq_forward(arr, len(ops), 0, fake, outs, ds, m, n, None)
+
+    ok = [(9, 0, 0, 1, 0.0), (1, 0, 1, 2, 0.0), (12, 2, 0, 0, 0.0)]            # swish: sigmoid, mul, out
+    assert run(ok) == 0
+    assert run([(99, 0, 0, 1, 0.0), (12, 1, 0, 0, 0.0)]) == 10                  # unknown opcode
+    assert run([(9, 3, 0, 1, 0.0), (12, 1, 0, 0, 0.0)]) == 10                   # reads a register never written
+    assert run([(9, 0, 0, 0, 0.0), (12, 0, 0, 0, 0.0)]) == 10                   # writes the source register
+    assert run([(9, 0, 0, 12, 0.0), (12, 1, 0, 0, 0.0)]) == 10                  # register out of range
+    assert run([(9, 0, 0, 1, 0.0)]) == 10                                       # no result produced
+    assert run([(9, 0, 0, 1, 0.0), (12, 1, 0, 1, 0.0)]) == 10                   # result slot out of range for m = 1
+    assert run(ok, m=5) == 10 and run(ok, m=0) == 10
+    assert lib.nfad_seq_forward(None, 3, 0, fake, outs, ds, 1, 0, None) == 3
+    assert run(ok * 11) == 10                                                    # more than 32 instructions
