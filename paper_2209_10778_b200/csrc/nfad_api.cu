@@ -104,6 +104,15 @@ cudaError_t noalloc_scratch(void** out)
     return cudaSuccess;
 }
 
+// [rows, cols] of the bias-fused entry points: cols must fit 31 bits, the element count a size_t of bytes.
+int check_shape(size_t rows, size_t cols, size_t* n)
+{
+    if (cols >= (size_t(1) << 31)) return NFAD_E_TOO_LARGE;
+    if (rows && cols > (~size_t(0) / 8) / rows) return NFAD_E_TOO_LARGE;
+    *n = rows * cols;
+    return NFAD_OK;
+}
+
 }  // namespace
 
 namespace nfad {
@@ -217,14 +226,6 @@ int nfad_probe_stream(int reads, int writes, const void* a, const void* b, void*
 }
 
 // ---- the pass fused with its producer's bias ----------------------------------------------
-
-static int check_shape(size_t rows, size_t cols, size_t* n)
-{
-    if (cols >= (size_t(1) << 31)) return NFAD_E_TOO_LARGE;
-    if (rows && cols > (~size_t(0) / 8) / rows) return NFAD_E_TOO_LARGE;     // rows * cols * element size must fit
-    *n = rows * cols;
-    return NFAD_OK;
-}
 
 int nfad_bias_act_forward(int kind, int dtype, const void* x, const void* bias, void* y, void* dfdx, size_t rows,
                           size_t cols, nfad_stream_t stream)
