@@ -71,7 +71,14 @@ cudaError_t seq_backward_t(const void* const* g, const void* const* d, int m, vo
     a.m = m;
     a.n = n;
     a.packets = al ? n / S::kVec : 0;
-    return launch_pdl(seq_backward_kernel<S>, grid_for(al ? a.packets : n), st, a);
+    const int u = seq_bwd_unroll(m);
+    const unsigned grid = grid_for(al ? (a.packets + u - 1) / u : 0);
+    switch (m) {
+    case 1: return launch_pdl(seq_backward_kernel<S, 1>, grid, st, a);
+    case 2: return launch_pdl(seq_backward_kernel<S, 2>, grid, st, a);
+    case 3: return launch_pdl(seq_backward_kernel<S, 3>, grid, st, a);
+    default: return launch_pdl(seq_backward_kernel<S, 4>, grid, st, a);
+    }
 }
 
 template <class S>

@@ -142,31 +142,56 @@ struct SeqBackwardArgs {
     size_t packets;    // whole 16-byte packets handled by the vector loop (0 unless every pointer is 16-byte aligned)
 };
 
-template <class S>
-__global__ void __launch_bounds__(kBlock) seq_backward_kernel(const SeqBackwardArgs a)
+// M is a template parameter so that all 2 M loads of a packet are issued before the first use; a CTA takes one
+// tile of kBlock * U packets, U = 2 for one or two results and 1 beyond (what 64 registers hold).
+constexpr int seq_bwd_unroll(int m) { return m <= 2 ? 2 : 1; }
+
+template <class S, int M>
+__global__ void __launch_bounds__(kBlock, 4) seq_backward_kernel(const SeqBackwardArgs a)
 {
     using E = typename S::elem;
     constexpr int V = S::kVec;
+    constexpr int U = seq_bwd_unroll(M);
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     asm volatile("griddepcontrol.wait;" ::: "memory");
-    for (size_t pk = size_t(blockIdx.x) * kBlock + threadIdx.x; pk < a.packets; pk += size_t(gridDim.x) * kBlock) {
-        float acc[V], gv[V], dv[V];
-        S::unpack(load_packet(static_cast<const uint4*>(a.g[0]) + pk), gv);
-        S::unpack(load_packet(static_cast<const uint4*>(a.d[0]) + pk), dv);
+    const size_t tile = size_t(kBlock) * U;
+    for (size_t base = size_t(blockIdx.x) * tile + threadIdx.x; base < a.packets; base += size_t(gridDim.x) * tile) {
+        uint4 rg[U][M], rd[U][M];
 #pragma unroll
-        for (int e = 0; e < V; ++e) acc[e] = gv[e] * dv[e];
-        for (int k = 1; k < a.m; ++k) {
-            S::unpack(load_packet(static_cast<const uint4*>(a.g[k]) + pk), gv);
-            S::unpack(load_packet(static_cast<const uint4*>(a.d[k]) + pk), dv);
+        for (int u = 0; u < U; ++u) {
+            const size_t pk = base + size_t(u) * kBlock;
+            if (pk < a.packets) {
 #pragma unroll
-            for (int e = 0; e < V; ++e) acc[e] = fmaf(gv[e], dv[e], acc[e]);
+                for (int k = 0; k < M; ++k) {
+                    rg[u][k] = load_packet(static_cast<const uint4*>(a.g[k]) + pk);
+                    rd[u][k] = load_packet(static_cast<const uint4*>(a.d[k]) + pk);
+                }
+            }
         }
-        *(static_cast<uint4*>(a.gin) + pk) = S::pack(acc);
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const size_t pk = base + size_t(u) * kBlock;
+            if (pk >= a.packets) continue;
+            float acc[V], gv[V], dv[V];
+            S::unpack(rg[u][0], gv);
+            S::unpack(rd[u][0], dv);
+#pragma unroll
+            for (int e = 0; e < V; ++e) acc[e] = gv[e] * dv[e];
+#pragma unroll
+            for (int k = 1; k < M; ++k) {
+                S::unpack(rg[u][k], gv);
+                S::unpack(rd[u][k], dv);
+#pragma unroll
+                for (int e = 0; e < V; ++e) acc[e] = fmaf(gv[e], dv[e], acc[e]);
+            }
+            *(static_cast<uint4*>(a.gin) + pk) = S::pack(acc);
+        }
     }
     if (blockIdx.x == 0) {
         for (size_t i = a.packets * V + threadIdx.x; i < a.n; i += kBlock) {
             float acc = S::load1(static_cast<const E*>(a.g[0]) + i) * S::load1(static_cast<const E*>(a.d[0]) + i);
-            for (int k = 1; k < a.m; ++k)
+#pragma unroll
+            for (int k = 1; k < M; ++k)
                 acc = fmaf(S::load1(static_cast<const E*>(a.g[k]) + i), S::load1(static_cast<const E*>(a.d[k]) + i), acc);
             S::store1(static_cast<E*>(a.gin) + i, acc);
         }
