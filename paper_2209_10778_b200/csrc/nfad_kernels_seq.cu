@@ -93,7 +93,16 @@ cudaError_t ew_t(int op, int backward, float c, const void* const* in, void* con
     a.c = c;
     a.n = n;
     a.packets = al ? n / S::kVec : 0;
-    return launch_pdl(ew_kernel<S>, grid_for(al ? a.packets : n), st, a);
+    const unsigned grid = grid_for(al ? (a.packets + kEwUnroll - 1) / kEwUnroll : 0);
+#define NFAD_EW_CASE(OPC) \
+    case OPC: return backward ? launch_pdl(ew_kernel<S, OPC, true>, grid, st, a) : launch_pdl(ew_kernel<S, OPC, false>, grid, st, a);
+    switch (op) {
+        NFAD_EW_CASE(kSeqAdd) NFAD_EW_CASE(kSeqMul) NFAD_EW_CASE(kSeqScale) NFAD_EW_CASE(kSeqAddConst) NFAD_EW_CASE(kSeqExp)
+        NFAD_EW_CASE(kSeqLog1p) NFAD_EW_CASE(kSeqTanh) NFAD_EW_CASE(kSeqErf) NFAD_EW_CASE(kSeqSoftplus) NFAD_EW_CASE(kSeqSigmoid)
+        NFAD_EW_CASE(kSeqHalfOnePlusTanh) NFAD_EW_CASE(kSeqHalfOnePlusErf)
+    }
+#undef NFAD_EW_CASE
+    return cudaErrorInvalidValue;
 }
 
 }  // namespace

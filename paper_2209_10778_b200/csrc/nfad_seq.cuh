@@ -144,7 +144,7 @@ struct SeqBackwardArgs {
 
 // M is a template parameter so that all 2 M loads of a packet are issued before the first use; a CTA takes one
 // tile of kBlock * U packets, U = 2 for one or two results and 1 beyond (what 64 registers hold).
-constexpr int seq_bwd_unroll(int m) { return m <= 2 ? 2 : 1; }
+__host__ __device__ constexpr int seq_bwd_unroll(int m) { return m <= 2 ? 2 : 1; }
 
 template <class S, int M>
 __global__ void __launch_bounds__(kBlock, 4) seq_backward_kernel(const SeqBackwardArgs a)
@@ -253,22 +253,44 @@ __device__ __forceinline__ void ew_apply(int op, int backward, float c, float i0
     }
 }
 
-template <class S>
-__global__ void __launch_bounds__(kBlock) ew_kernel(const EwArgs a)
+// (Tiled like the other kernels -- two packets per thread, every load issued before the first use -- so that the
+// operator-by-operator comparator runs each operator at the bandwidth a framework's own element-wise kernel reaches.)
+constexpr int kEwUnroll = 2;
+
+// OP and BWD are template parameters: each operator gets its own specialised kernel, as in a framework.
+template <class S, int OP, bool BWD>
+__global__ void __launch_bounds__(kBlock, 4) ew_kernel(const EwArgs a)
 {
     using E = typename S::elem;
     constexpr int V = S::kVec;
+    constexpr int U = kEwUnroll;
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     asm volatile("griddepcontrol.wait;" ::: "memory");
-    for (size_t pk = size_t(blockIdx.x) * kBlock + threadIdx.x; pk < a.packets; pk += size_t(gridDim.x) * kBlock) {
-        float i0[V], i1[V], i2[V], o0[V], o1[V];
-        S::unpack(load_packet(static_cast<const uint4*>(a.in[0]) + pk), i0);
-        if (a.in[1]) S::unpack(load_packet(static_cast<const uint4*>(a.in[1]) + pk), i1);
-        if (a.in[2]) S::unpack(load_packet(static_cast<const uint4*>(a.in[2]) + pk), i2);
+    const size_t tile = size_t(kBlock) * U;
+    for (size_t base = size_t(blockIdx.x) * tile + threadIdx.x; base < a.packets; base += size_t(gridDim.x) * tile) {
+        uint4 r0[U], r1[U], r2[U];
 #pragma unroll
-        for (int e = 0; e < V; ++e) ew_apply(a.op, a.backward, a.c, i0[e], a.in[1] ? i1[e] : 0.0f, a.in[2] ? i2[e] : 0.0f, o0[e], o1[e]);
-        *(static_cast<uint4*>(a.out[0]) + pk) = S::pack(o0);
-        if (a.out[1]) *(static_cast<uint4*>(a.out[1]) + pk) = S::pack(o1);
+        for (int u = 0; u < U; ++u) {
+            const size_t pk = base + size_t(u) * kBlock;
+            if (pk < a.packets) {
+                r0[u] = load_packet(static_cast<const uint4*>(a.in[0]) + pk);
+                if (a.in[1]) r1[u] = load_packet(static_cast<const uint4*>(a.in[1]) + pk);
+                if (a.in[2]) r2[u] = load_packet(static_cast<const uint4*>(a.in[2]) + pk);
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const size_t pk = base + size_t(u) * kBlock;
+            if (pk >= a.packets) continue;
+            float i0[V], i1[V], i2[V], o0[V], o1[V];
+            S::unpack(r0[u], i0);
+            if (a.in[1]) S::unpack(r1[u], i1);
+            if (a.in[2]) S::unpack(r2[u], i2);
+#pragma unroll
+            for (int e = 0; e < V; ++e) ew_apply(OP, BWD, a.c, i0[e], a.in[1] ? i1[e] : 0.0f, a.in[2] ? i2[e] : 0.0f, o0[e], o1[e]);
+            *(static_cast<uint4*>(a.out[0]) + pk) = S::pack(o0);
+            if (a.out[1]) *(static_cast<uint4*>(a.out[1]) + pk) = S::pack(o1);
+        }
     }
     if (blockIdx.x == 0) {
         for (size_t i = a.packets * V + threadIdx.x; i < a.n; i += kBlock) {
@@ -276,7 +298,7 @@ __global__ void __launch_bounds__(kBlock) ew_kernel(const EwArgs a)
             float i1 = a.in[1] ? S::load1(static_cast<const E*>(a.in[1]) + i) : 0.0f;
             float i2 = a.in[2] ? S::load1(static_cast<const E*>(a.in[2]) + i) : 0.0f;
             float o0, o1;
-            ew_apply(a.op, a.backward, a.c, i0, i1, i2, o0, o1);
+            ew_apply(OP, BWD, a.c, i0, i1, i2, o0, o1);
             S::store1(static_cast<E*>(a.out[0]) + i, o0);
             if (a.out[1]) S::store1(static_cast<E*>(a.out[1]) + i, o1);
         }
