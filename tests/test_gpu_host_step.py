@@ -82,3 +82,25 @@ def test_host_step_refusals():
     assert lib.nfad_host_step(0, 0, p, p, p, None, p, 0, None, 0, 0, st) == 0
     assert lib.nfad_host_step(0, 0, p, p, p, None, p, 4096, ws.data_ptr(), 1 << 20, 2, st) == 8
     assert nfad.nfad_host_step_workspace_bytes(torch.float32, 0) == 0
+
+
+def test_host_step_inputs_ready_with_changing_workspaces():
+    # consecutive calls that may run ahead (inputs ready) but use different workspaces and chunk sizes: the second
+    # must not touch slots the first still uses, and each must give the device calls' bits
+    n1, n2 = 3 * (1 << 20) + 5, (1 << 19) + 3
+    x1, g1 = W.normal(n1, "bf16", 71, 1.0).pin_memory(), W.normal(n1, "bf16", 72, 1.0).pin_memory()
+    x2, g2 = W.normal(n2, "f32", 73, 1.0).pin_memory(), W.normal(n2, "f32", 74, 1.0).pin_memory()
+    y1, gi1 = torch.empty_like(x1).pin_memory(), torch.empty_like(x1).pin_memory()
+    y2, gi2 = torch.empty_like(x2).pin_memory(), torch.empty_like(x2).pin_memory()
+    ws1 = torch.empty(nfad.nfad_host_step_workspace_bytes(torch.bfloat16, n1), dtype=torch.uint8, device=DEV)
+    ws2 = torch.empty(4 * 5 * 4096 * 4, dtype=torch.uint8, device=DEV)          # small: many chunks
+    nfad.nfad_host_step("mish", x1, g1, y1, None, gi1, ws1, inputs_ready=True)
+    nfad.nfad_host_step("swish", x2, g2, y2, None, gi2, ws2, inputs_ready=True)
+    nfad.nfad_host_step("gelu_erf", x1, g1, y1, None, gi1, ws1, inputs_ready=True)   # back to the first layout
+    torch.cuda.synchronize()
+    for kind, x, g, y, gi in (("gelu_erf", x1, g1, y1, gi1), ("swish", x2, g2, y2, gi2)):
+        xd, gd = x.to(DEV), g.to(DEV)
+        yd, dd, gid = torch.empty_like(xd), torch.empty_like(xd), torch.empty_like(xd)
+        nfad.nfad_act_forward(kind, xd, yd, dd)
+        nfad.nfad_act_backward(kind, gd, dd, gid)
+        assert np.array_equal(W.raw_numpy(y), W.raw_numpy(yd)) and np.array_equal(W.raw_numpy(gi), W.raw_numpy(gid))

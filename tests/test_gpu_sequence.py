@@ -229,3 +229,32 @@ def test_malformed_programs_are_refused():
             nfad.nfad_seq_forward(prog, x, [y], [d])
         assert e.value.status == 10
     torch.cuda.synchronize()
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_four_results_forward_and_backward(dtype, executor):
+    # one source, four results (the most the interface takes): x^2, sigmoid(x), tanh(x) * x, exp(-|..|)-free softplus(x)
+    p = sequence.FadProgram()
+    x = p.x()
+    p.output(p.mul(x, x))
+    p.output(p.unary("sigmoid", x))
+    p.output(p.mul(p.unary("tanh", x), x))
+    p.output(p.unary("softplus", x))
+    n = 40003
+    xt = (W.normal(n, "f32", 15, 1.5, DEV).clamp_(-6, 6)).to(W.TORCH_DTYPES[dtype])
+    ys, ds = sequence.run_fused(p, xt)
+    assert nfad.nfad_seq_last_executor() == executor
+    gs = [W.normal(n, dtype, 20 + k, 1.0, DEV) for k in range(4)]
+    gin = sequence.backward_fused(gs, ds)
+    torch.cuda.synchronize()
+    x64 = oracle.widen(dtype, W.raw_numpy(xt))
+    y, d = oracle.seq_forward(p.ops, x64, 4)
+    for k in range(4):
+        assert _close(dtype, ys[k], y[k], x64).all(), ("value", k)
+        assert _close(dtype, ds[k], d[k], x64).all(), ("derivative", k)
+    g64 = np.stack([oracle.widen(dtype, W.raw_numpy(g)) for g in gs])
+    d_saved = np.stack([oracle.widen(dtype, W.raw_numpy(t)) for t in ds])
+    want, want_abs = oracle.seq_backward(g64, d_saved)
+    got = oracle.widen(dtype, W.raw_numpy(gin))
+    tol = (2.0 ** -22 if dtype == "f32" else 2.0 ** -7) * want_abs + 1e-30
+    assert (np.abs(got - want) <= tol).all()
