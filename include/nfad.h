@@ -26,6 +26,10 @@
  *   - Work is enqueued on `stream` (a cudaStream_t; 0 is the legacy default
  *     stream) of the current device and the call returns at once.  The return
  *     value covers argument validation and the launch, not completion.
+ *   - The entry points that take device pointers only enqueue kernels (no allocation, no
+ *     synchronisation, no host-side wait) and can be captured into a CUDA graph; the exceptions
+ *     (nfad_host_step; the first call of a new run-time sequence when it is compiled; the first
+ *     nfad_cmp_recompute_backward_noalloc on a device) say so where they are declared.
  *   - n == 0 is valid and does nothing.  n is 64-bit: 2^30 fp32 elements and
  *     beyond are indexed correctly.
  *   - Return value: an nfad_status.  Nothing aborts or traps.  After
