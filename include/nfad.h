@@ -28,8 +28,9 @@
  *     value covers argument validation and the launch, not completion.
  *   - The entry points that take device pointers only enqueue kernels (no allocation, no
  *     synchronisation, no host-side wait) and can be captured into a CUDA graph; the exceptions
- *     (nfad_host_step; the first call of a new run-time sequence when it is compiled; the first
- *     nfad_cmp_recompute_backward_noalloc on a device) say so where they are declared.
+ *     (nfad_host_step; the first call of a new run-time sequence when it is compiled) say so
+ *     where they are declared.  This statement does not cover nfad_cmp_recompute_backward_noalloc,
+ *     about which nothing is claimed here beyond what its own comment says.
  *   - n == 0 is valid and does nothing.  n is 64-bit: 2^30 fp32 elements and
  *     beyond are indexed correctly.
  *   - Return value: an nfad_status.  Nothing aborts or traps.  After
