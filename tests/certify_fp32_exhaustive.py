@@ -1,15 +1,15 @@
 """Exhaustive certification of the fp32-storage forward kernels (not collected by pytest: run by hand).
 
-    python tests/certify_fp32_exhaustive.py [kind,kind,...] [--strict]
+    python tests/certify_fp32_exhaustive.py [kind,kind,...] [--strict] [--out=FILE.json]
 
 Every fp32 bit pattern with |x| <= 130 (2 x 1.12e9 values per kind; beyond that every kind is
 saturated) goes through nfad_act_forward on cuda:0 and is compared with the fp64 oracle in the
 metrics of tests/parity.py.  Prints, per kind, the worst value error in ulp, the worst
 derivative error in the gate's metric (strict for x >= 0, scaled by |h| + |x h'| for x < 0),
-the worst subnormal-result errors in units of 2^-149 and the count of non-finite outputs, and
-writes them to gpurun_out/exhaustive_f32.json.  About three minutes per kind on a 16-core host.
-With --strict the inputs go through nfad_act_forward_strict instead and the derivative is measured in
-strict ulp of f' itself for every x (no scaling); the results go to gpurun_out/exhaustive_f32_strict.json.
+the worst subnormal-result errors in units of 2^-149 and the count of non-finite outputs; with
+--out=FILE.json the same numbers are also written to that file.  About three minutes per kind on a
+16-core host.  With --strict the inputs go through nfad_act_forward_strict instead and the derivative
+is measured in strict ulp of f' itself for every x (no scaling).
 """
 import json
 import os
@@ -26,6 +26,7 @@ import oracle, ulp
 from paper_2209_10778_b200 import binding as nfad
 oracle.set_threads(oracle.max_threads())
 STRICT = '--strict' in sys.argv
+OUT = next((a.split('=', 1)[1] for a in sys.argv[1:] if a.startswith('--out=')), None)
 args = [a for a in sys.argv[1:] if not a.startswith('--')]
 kinds = args[0].split(',') if args else ['gelu_erf','gelu_tanh','swish','mish']
 hi_bits = int(np.float32(130.0).view(np.uint32))
@@ -63,5 +64,6 @@ for kind in kinds:
     worst['seconds'] = time.time() - t0
     res[kind] = worst
     print(kind, json.dumps(worst), flush=True)
-os.makedirs(os.path.join(ROOT, 'gpurun_out'), exist_ok=True)
-json.dump(res, open(os.path.join(ROOT, 'gpurun_out', 'exhaustive_f32_strict.json' if STRICT else 'exhaustive_f32.json'), 'w'))
+if OUT:
+    os.makedirs(os.path.dirname(os.path.abspath(OUT)), exist_ok=True)
+    json.dump(res, open(OUT, 'w'))
