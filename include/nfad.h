@@ -257,6 +257,10 @@ NFAD_API int nfad_seq_forward(const nfad_seq_op* program, int n_ops, int dtype, 
 NFAD_API int nfad_seq_set_executor(int mode);
 NFAD_API int nfad_seq_last_executor(void);
 NFAD_API const char* nfad_seq_compile_log(void);
+/* The CUDA source the compiled executor builds for a sequence (valid until the calling thread's next call of this
+ * function); NULL for a malformed program or a bad dtype.  Needs no device: for inspection and for testing the
+ * generator where no GPU is present. */
+NFAD_API const char* nfad_seq_compiled_source(const nfad_seq_op* program, int n_ops, int dtype, int m);
 
 /*
  * Backward of a sequence with m results (Section II-E; for a binary merge "the post-process

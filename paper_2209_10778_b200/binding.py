@@ -33,7 +33,7 @@ EXPORTS = (
     "nfad_bias_act_forward", "nfad_bias_act_backward", "nfad_bias_act_backward_scratch_bytes",
     "nfad_act_forward_strict",
     "nfad_host_step", "nfad_host_step_workspace_bytes",
-    "nfad_seq_set_executor", "nfad_seq_last_executor", "nfad_seq_compile_log",
+    "nfad_seq_set_executor", "nfad_seq_last_executor", "nfad_seq_compile_log", "nfad_seq_compiled_source",
 )
 OPCODES = {"add": 0, "mul": 1, "scale": 2, "add_const": 3, "exp": 4, "log1p": 5, "tanh": 6, "erf": 7, "softplus": 8,
            "sigmoid": 9, "half_one_plus_tanh": 10, "half_one_plus_erf": 11, "out": 12}
@@ -92,6 +92,8 @@ def load() -> ctypes.CDLL:
         lib.nfad_seq_set_executor.restype = ci
         lib.nfad_seq_last_executor.argtypes = []
         lib.nfad_seq_last_executor.restype = ci
+        lib.nfad_seq_compiled_source.argtypes = [ctypes.POINTER(SeqOp), ci, ci, ci]
+        lib.nfad_seq_compiled_source.restype = ctypes.c_char_p
         lib.nfad_seq_compile_log.argtypes = []
         lib.nfad_seq_compile_log.restype = ctypes.c_char_p
         lib.nfad_host_step.argtypes = [ci, ci, vp, vp, vp, vp, vp, sz, vp, sz, ci, vp]
@@ -325,9 +327,7 @@ def _ptr_array(tensors, name, like):
     return arr
 
 
-def nfad_seq_forward(program, x: torch.Tensor, ys, dfdxs) -> None:
-    """Runs a FAD sequence (a list of SeqOp, or of (op, a, b, dst, c) tuples with op a name or code)
-    on x in one kernel: ys[k] = k-th result, dfdxs[k] = its derivative with respect to x."""
+def _seq_ops(program):
     ops = (SeqOp * len(program))()
     for i, o in enumerate(program):
         if isinstance(o, SeqOp):
@@ -335,6 +335,20 @@ def nfad_seq_forward(program, x: torch.Tensor, ys, dfdxs) -> None:
         else:
             op, a, b, dst, c = o
             ops[i] = SeqOp(OPCODES[op] if isinstance(op, str) else int(op), int(a), int(b), int(dst), float(c))
+    return ops
+
+
+def nfad_seq_compiled_source(program, dtype, m: int) -> Optional[str]:
+    """The CUDA source the compiled executor builds for this sequence (no device needed); None if malformed."""
+    code = _TORCH_TO_CODE[dtype] if isinstance(dtype, torch.dtype) else DTYPES[dtype]
+    text = load().nfad_seq_compiled_source(_seq_ops(program), len(program), code, int(m))
+    return text.decode() if text is not None else None
+
+
+def nfad_seq_forward(program, x: torch.Tensor, ys, dfdxs) -> None:
+    """Runs a FAD sequence (a list of SeqOp, or of (op, a, b, dst, c) tuples with op a name or code)
+    on x in one kernel: ys[k] = k-th result, dfdxs[k] = its derivative with respect to x."""
+    ops = _seq_ops(program)
     px = _tensor(x, "x")
     if len(ys) != len(dfdxs):
         raise ValueError("ys and dfdxs must have the same length")

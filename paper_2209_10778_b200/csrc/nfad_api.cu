@@ -3,6 +3,7 @@
 #include <stdint.h>
 
 #include <mutex>
+#include <string>
 
 #include "../../include/nfad.h"
 #include "nfad_internal.h"
@@ -325,13 +326,13 @@ int nfad_cmp_recompute_backward_noalloc(int kind, int dtype, const void* grad_ou
     return nfad_cmp_recompute_backward(kind, dtype, grad_out, x, scratch, NFAD_NOALLOC_SCRATCH_BYTES, grad_in, n, stream);
 }
 
-int nfad_seq_forward(const nfad_seq_op* program, int n_ops, int dtype, const void* x, void* const* y, void* const* dfdx,
-                     int m, size_t n, nfad_stream_t stream)
+// Validates a sequence and copies it into the launcher's form.
+static int parse_program(const nfad_seq_op* program, int n_ops, int m, nfad::SeqProgramHost* out)
 {
-    if (dtype < 0 || dtype > 2) return NFAD_E_DTYPE;
-    if (!program || !y || !dfdx) return NFAD_E_NULL;
+    if (!program) return NFAD_E_NULL;
     if (n_ops < 1 || n_ops > nfad::kSeqMaxOpsHost || m < 1 || m > 4) return NFAD_E_PROGRAM;
-    nfad::SeqProgramHost p = {};
+    nfad::SeqProgramHost& p = *out;
+    p = nfad::SeqProgramHost{};
     p.n_ops = n_ops;
     constexpr int kRegs = 12;
     bool written[kRegs] = {true};
@@ -352,6 +353,28 @@ int nfad_seq_forward(const nfad_seq_op* program, int n_ops, int dtype, const voi
         p.op[i] = o.op; p.a[i] = o.a; p.b[i] = binary ? o.b : o.a; p.dst[i] = o.dst; p.c[i] = o.c;
     }
     for (int k = 0; k < m; ++k) if (!produced[k]) return NFAD_E_PROGRAM;
+    return NFAD_OK;
+}
+
+const char* nfad_seq_compiled_source(const nfad_seq_op* program, int n_ops, int dtype, int m)
+{
+    static thread_local std::string text;
+    nfad::SeqProgramHost p;
+    if (dtype < 0 || dtype > 2 || parse_program(program, n_ops, m, &p) != NFAD_OK) return nullptr;
+    text = nfad::seq_generate_source(p, dtype, m);
+    return text.c_str();
+}
+
+int nfad_seq_forward(const nfad_seq_op* program, int n_ops, int dtype, const void* x, void* const* y, void* const* dfdx,
+                     int m, size_t n, nfad_stream_t stream)
+{
+    if (dtype < 0 || dtype > 2) return NFAD_E_DTYPE;
+    if (!program || !y || !dfdx) return NFAD_E_NULL;
+    nfad::SeqProgramHost p;
+    {
+        int prc = parse_program(program, n_ops, m, &p);
+        if (prc) return prc;
+    }
     const void* in[1] = {x};
     void* out[8];
     for (int k = 0; k < m; ++k) { out[k] = y[k]; out[m + k] = dfdx[k]; }

@@ -6,6 +6,8 @@
 #include <cuda_runtime.h>
 #include <stddef.h>
 
+#include <string>
+
 namespace nfad {
 
 enum Kind { kGeluErf = 0, kGeluTanh = 1, kSwish = 2, kMish = 3 };
@@ -43,6 +45,7 @@ void seq_set_executor_mode(int mode);
 int seq_last_executor();                 // of the calling thread: 0 none yet, 1 interpreter, 2 compiled
 void seq_note_executor(int which);
 const char* seq_jit_log();
+std::string seq_generate_source(const SeqProgramHost& p, int dtype, int m);   // what the compiled executor would compile
 cudaError_t launch_seq_backward(int dtype, const void* const* g, const void* const* d, int m, void* gin, size_t n, cudaStream_t st);
 cudaError_t launch_ew(int op, int backward, float c, int dtype, const void* const* in, void* const* out, size_t n, cudaStream_t st);
 

@@ -171,6 +171,11 @@ cudaError_t build(const std::string& src, int dev, CUfunction* out)
 
 }  // namespace
 
+std::string seq_generate_source(const SeqProgramHost& p, int dtype, int m)
+{
+    return generate(p, m, dtype == kF32 ? "StoreF32" : dtype == kBF16 ? "StoreBF16" : "StoreF16");
+}
+
 int seq_executor_mode() { return g_mode; }
 void seq_set_executor_mode(int mode) { std::lock_guard<std::mutex> lock(g_mutex); g_mode = mode; }
 int seq_last_executor() { return g_last_executor; }
