@@ -323,6 +323,10 @@ NFAD_API int nfad_ew_op(int op, int backward, float c, int dtype, const void* in
  */
 NFAD_API int nfad_bias_act_forward(int kind, int dtype, const void* x, const void* bias, void* y, void* dfdx, size_t rows,
                                    size_t cols, nfad_stream_t stream);
+/* The value-only form (a pass that will not be differentiated): y = f(x + bias), bit-identical to the y of
+ * nfad_bias_act_forward; no dfdx. */
+NFAD_API int nfad_bias_act_forward_infer(int kind, int dtype, const void* x, const void* bias, void* y, size_t rows,
+                                         size_t cols, nfad_stream_t stream);
 NFAD_API int nfad_bias_act_backward(int kind, int dtype, const void* grad_out, const void* dfdx, void* grad_in,
                                     float* grad_bias, void* scratch, size_t scratch_bytes, size_t rows, size_t cols,
                                     nfad_stream_t stream);

@@ -30,7 +30,7 @@ EXPORTS = (
     "nfad_saved_bytes_per_element", "nfad_last_cuda_error", "nfad_status_string", "nfad_version",
     "nfad_probe_stream", "nfad_cmp_recompute_backward_noalloc",
     "nfad_seq_forward", "nfad_seq_backward", "nfad_ew_op",
-    "nfad_bias_act_forward", "nfad_bias_act_backward", "nfad_bias_act_backward_scratch_bytes",
+    "nfad_bias_act_forward", "nfad_bias_act_forward_infer", "nfad_bias_act_backward", "nfad_bias_act_backward_scratch_bytes",
     "nfad_act_forward_strict",
     "nfad_host_step", "nfad_host_step_workspace_bytes",
     "nfad_seq_set_executor", "nfad_seq_last_executor", "nfad_seq_compile_log", "nfad_seq_compiled_source",
@@ -84,6 +84,8 @@ def load() -> ctypes.CDLL:
         lib.nfad_ew_op.restype = ci
         lib.nfad_bias_act_forward.argtypes = [ci, ci, vp, vp, vp, vp, sz, sz, vp]
         lib.nfad_bias_act_forward.restype = ci
+        lib.nfad_bias_act_forward_infer.argtypes = [ci, ci, vp, vp, vp, sz, sz, vp]
+        lib.nfad_bias_act_forward_infer.restype = ci
         lib.nfad_bias_act_backward.argtypes = [ci, ci, vp, vp, vp, vp, vp, sz, sz, sz, vp]
         lib.nfad_bias_act_backward.restype = ci
         lib.nfad_bias_act_backward_scratch_bytes.argtypes = [ci, sz, sz]
@@ -257,6 +259,18 @@ def nfad_bias_act_forward(kind, x: torch.Tensor, bias: torch.Tensor, y: torch.Te
     with _on_device(x.device):
         _check(load().nfad_bias_act_forward(_kind(kind), _TORCH_TO_CODE[x.dtype], px, pb, _tensor(y, "y", x),
                                             _tensor(dfdx, "dfdx", x), rows, cols, _stream(x)), "nfad_bias_act_forward")
+
+
+def nfad_bias_act_forward_infer(kind, x: torch.Tensor, bias: torch.Tensor, y: torch.Tensor) -> None:
+    """y = f(x + bias): the value-only form of nfad_bias_act_forward."""
+    px = _tensor(x, "x")
+    if bias.dtype != x.dtype or bias.device != x.device:
+        raise ValueError("bias must match x's dtype and device")
+    pb = _tensor(bias, "bias")
+    rows, cols = _rows_cols(x, bias.numel())
+    with _on_device(x.device):
+        _check(load().nfad_bias_act_forward_infer(_kind(kind), _TORCH_TO_CODE[x.dtype], px, pb, _tensor(y, "y", x), rows, cols,
+                                                  _stream(x)), "nfad_bias_act_forward_infer")
 
 
 def nfad_bias_act_backward_scratch_bytes(dtype, rows: int, cols: int, device=None) -> int:

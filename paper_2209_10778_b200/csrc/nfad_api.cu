@@ -228,8 +228,9 @@ int nfad_probe_stream(int reads, int writes, const void* a, const void* b, void*
 
 // ---- the pass fused with its producer's bias ----------------------------------------------
 
-int nfad_bias_act_forward(int kind, int dtype, const void* x, const void* bias, void* y, void* dfdx, size_t rows,
-                          size_t cols, nfad_stream_t stream)
+// dfdx == nullptr selects the value-only pass
+static int bias_forward_common(int kind, int dtype, const void* x, const void* bias, void* y, void* dfdx, bool train, size_t rows,
+                               size_t cols, nfad_stream_t stream)
 {
     if (kind < 0 || kind > 3) return NFAD_E_KIND;
     if (dtype < 0 || dtype > 2) return NFAD_E_DTYPE;
@@ -238,20 +239,33 @@ int nfad_bias_act_forward(int kind, int dtype, const void* x, const void* bias, 
     if (rc) return rc;
     const void* in[1] = {x};
     void* out[2] = {y, dfdx};
-    rc = check(kind, dtype, in, 1, out, 2, n);
+    rc = check(kind, dtype, in, 1, out, train ? 2 : 1, n);
     if (rc || n == 0) return rc;
     const size_t es = elem_size(dtype);
     if (!bias) return NFAD_E_NULL;
     if (reinterpret_cast<uintptr_t>(bias) % es) return NFAD_E_ALIGN;
-    if (overlaps(bias, y, cols * es, n * es) || overlaps(bias, dfdx, cols * es, n * es)) return NFAD_E_OVERLAP;
+    if (overlaps(bias, y, cols * es, n * es) || (train && overlaps(bias, dfdx, cols * es, n * es))) return NFAD_E_OVERLAP;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    cudaError_t e = dtype == NFAD_F32 ? nfad::launch_bias_forward_f32(kind, x, bias, y, dfdx, rows, cols, st)
-                                      : nfad::launch_bias_forward_16(kind, dtype, x, bias, y, dfdx, rows, cols, st);
+    void* d = train ? dfdx : nullptr;
+    cudaError_t e = dtype == NFAD_F32 ? nfad::launch_bias_forward_f32(kind, x, bias, y, d, rows, cols, st)
+                                      : nfad::launch_bias_forward_16(kind, dtype, x, bias, y, d, rows, cols, st);
     if (e != cudaSuccess) {
         g_last_cuda_error = static_cast<int>(e);
         return NFAD_E_CUDA;
     }
     return NFAD_OK;
+}
+
+int nfad_bias_act_forward(int kind, int dtype, const void* x, const void* bias, void* y, void* dfdx, size_t rows,
+                          size_t cols, nfad_stream_t stream)
+{
+    return bias_forward_common(kind, dtype, x, bias, y, dfdx, true, rows, cols, stream);
+}
+
+int nfad_bias_act_forward_infer(int kind, int dtype, const void* x, const void* bias, void* y, size_t rows, size_t cols,
+                                nfad_stream_t stream)
+{
+    return bias_forward_common(kind, dtype, x, bias, y, nullptr, false, rows, cols, stream);
 }
 
 size_t nfad_bias_act_backward_scratch_bytes(int dtype, size_t rows, size_t cols)

@@ -82,7 +82,8 @@ struct BiasForwardArgs {
 // z = x + b, one fp32 addition that the compiler may not merge into anything
 __device__ __forceinline__ float bias_sum(float x, float b) { return __fadd_rn(x, b); }
 
-template <class S, class K, class P>
+// kTrain: y and f'; otherwise y alone (d is not touched)
+template <class S, class K, class P, bool kTrain>
 __device__ __forceinline__ void bias_forward_packet(const uint4& rx, const float (&vb)[S::kVec], uint4* y, uint4* d)
 {
     constexpr int V = S::kVec;
@@ -90,16 +91,20 @@ __device__ __forceinline__ void bias_forward_packet(const uint4& rx, const float
     S::unpack(rx, vx);
 #pragma unroll
     for (int e = 0; e < V; ++e) {
-        ActOut o = evaluate<K, P>(bias_sum(vx[e], vb[e]));
-        vy[e] = o.y;
-        vd[e] = o.dydx;
+        if (kTrain) {
+            ActOut o = evaluate<K, P>(bias_sum(vx[e], vb[e]));
+            vy[e] = o.y;
+            vd[e] = o.dydx;
+        } else {
+            vy[e] = evaluate_value(K{}, P{}, bias_sum(vx[e], vb[e]));
+        }
     }
     store_packet<true>(y, S::pack(vy));
-    store_packet<false>(d, S::pack(vd));
+    if (kTrain) store_packet<false>(d, S::pack(vd));
 }
 
 // Vector path: cols a multiple of the packet size and every pointer 16-byte aligned.
-template <class S, class K, class P>
+template <class S, class K, class P, bool kTrain>
 __global__ void __launch_bounds__(kBiasMaxBlock, S::kMinBlocks) bias_forward_kernel(const BiasForwardArgs a)
 {
     constexpr int V = S::kVec;
@@ -125,35 +130,42 @@ __global__ void __launch_bounds__(kBiasMaxBlock, S::kMinBlocks) bias_forward_ker
 #pragma unroll
             for (int u = 0; u < U; ++u) rx[u] = load_packet(x4 + pk0 + size_t(u) * rp);
 #pragma unroll
-            for (int u = 0; u < U; ++u) bias_forward_packet<S, K, P>(rx[u], vb, y4 + pk0 + size_t(u) * rp, d4 + pk0 + size_t(u) * rp);
+            for (int u = 0; u < U; ++u) bias_forward_packet<S, K, P, kTrain>(rx[u], vb, y4 + pk0 + size_t(u) * rp, d4 + pk0 + size_t(u) * rp);
         } else {
 #pragma unroll
             for (int u = 0; u < U; ++u)
                 if (r0 + u < a.rows) rx[u] = load_packet(x4 + pk0 + size_t(u) * rp);
 #pragma unroll
             for (int u = 0; u < U; ++u)
-                if (r0 + u < a.rows) bias_forward_packet<S, K, P>(rx[u], vb, y4 + pk0 + size_t(u) * rp, d4 + pk0 + size_t(u) * rp);
+                if (r0 + u < a.rows) bias_forward_packet<S, K, P, kTrain>(rx[u], vb, y4 + pk0 + size_t(u) * rp, d4 + pk0 + size_t(u) * rp);
         }
     }
 }
 
 // Any cols, any (element-aligned) pointers: one element at a time, the same per-element code.
-template <class S, class K, class P>
+template <class S, class K, class P, bool kTrain>
 __global__ void __launch_bounds__(kBlock) bias_forward_scalar_kernel(const BiasForwardArgs a)
 {
     using E = typename S::elem;
     const size_t stride = size_t(gridDim.x) * kBlock;
     for (size_t i = size_t(blockIdx.x) * kBlock + threadIdx.x; i < a.n; i += stride) {
         const uint32_t c = uint32_t(i % a.cols);
-        ActOut o = evaluate<K, P>(bias_sum(S::load1(static_cast<const E*>(a.x) + i), S::load1(static_cast<const E*>(a.bias) + c)));
-        S::store1(static_cast<E*>(a.y) + i, o.y);
-        S::store1(static_cast<E*>(a.d) + i, o.dydx);
+        const float z = bias_sum(S::load1(static_cast<const E*>(a.x) + i), S::load1(static_cast<const E*>(a.bias) + c));
+        if (kTrain) {
+            ActOut o = evaluate<K, P>(z);
+            S::store1(static_cast<E*>(a.y) + i, o.y);
+            S::store1(static_cast<E*>(a.d) + i, o.dydx);
+        } else {
+            S::store1(static_cast<E*>(a.y) + i, evaluate_value(K{}, P{}, z));
+        }
     }
 }
 
+// d == nullptr: the value-only pass
 template <class S, class K, class P>
 cudaError_t launch_bias_forward(const void* x, const void* bias, void* y, void* d, size_t rows, size_t cols, cudaStream_t st)
 {
+    const bool train = d != nullptr;
     constexpr int V = S::kVec;
     BiasForwardArgs a;
     a.x = x; a.bias = bias; a.y = y; a.d = d;
@@ -164,7 +176,7 @@ cudaError_t launch_bias_forward(const void* x, const void* bias, void* y, void* 
     DeviceInfo di;
     cudaError_t e = device_info(&di);
     if (e != cudaSuccess) return e;
-    const bool vec = cols % V == 0 && aligned16(x) && aligned16(bias) && aligned16(y) && aligned16(d);
+    const bool vec = cols % V == 0 && aligned16(x) && aligned16(bias) && aligned16(y) && (!train || aligned16(d));
     cudaLaunchConfig_t cfg;
     cudaLaunchAttribute attr[1];
     if (!vec) {
@@ -172,7 +184,8 @@ cudaError_t launch_bias_forward(const void* x, const void* bias, void* y, void* 
         size_t blocks = (a.n + kBlock - 1) / kBlock;
         size_t cap = size_t(di.sm_count) * 8;
         bias_launch_config(&cfg, attr, blocks < cap ? blocks : cap, kBlock, st, false);
-        return cudaLaunchKernelEx(&cfg, bias_forward_scalar_kernel<S, K, P>, a);
+        return train ? cudaLaunchKernelEx(&cfg, bias_forward_scalar_kernel<S, K, P, true>, a)
+                     : cudaLaunchKernelEx(&cfg, bias_forward_scalar_kernel<S, K, P, false>, a);
     }
     a.row_packets = uint32_t(cols / V);
     const unsigned block = bias_block(a.row_packets);
@@ -180,7 +193,8 @@ cudaError_t launch_bias_forward(const void* x, const void* bias, void* y, void* 
     a.work = (rows + kBiasRows - 1) / kBiasRows;
     bias_launch_config(&cfg, attr, a.strips, block, st, true);
     cfg.gridDim.y = (unsigned)(a.work < 65535 ? a.work : 65535);
-    return cudaLaunchKernelEx(&cfg, bias_forward_kernel<S, K, P>, a);
+    return train ? cudaLaunchKernelEx(&cfg, bias_forward_kernel<S, K, P, true>, a)
+                 : cudaLaunchKernelEx(&cfg, bias_forward_kernel<S, K, P, false>, a);
 }
 
 // ---------------------------------------------------------------- backward with the bias gradient

@@ -252,3 +252,23 @@ def test_tall_narrow_tensor_covers_the_row_chunk_loop():
     # more row chunks than one grid dimension holds (rows / 4 > 65535): the forward kernel's chunk loop, and a backward
     # whose strips are narrower than one warp-wide access
     _run("swish", "bf16", 300000, 64, 55)
+
+
+@pytest.mark.parametrize("dtype", DTYPES)
+def test_value_only_forward_gives_the_training_value(dtype):
+    for rows, cols in ((300, 768), (41, 1003)):
+        x = W.normal(rows * cols, dtype, 81, 1.5, DEV)
+        bias = W.normal(cols, dtype, 82, 0.5, DEV)
+        for kind in KINDS:
+            y, d, yi = torch.empty_like(x), torch.empty_like(x), torch.full_like(x, 3.0)
+            nfad.nfad_bias_act_forward(kind, x, bias, y, d)
+            nfad.nfad_bias_act_forward_infer(kind, x, bias, yi)
+            torch.cuda.synchronize()
+            assert np.array_equal(W.raw_numpy(y), W.raw_numpy(yi)), (kind, dtype, rows, cols)
+    xs = torch.tensor([float("inf"), float("-inf"), float("nan"), 0.0], device=DEV, dtype=W.TORCH_DTYPES[dtype])
+    b1 = torch.zeros(4, device=DEV, dtype=W.TORCH_DTYPES[dtype])
+    out = torch.empty_like(xs)
+    for kind in KINDS:
+        nfad.nfad_bias_act_forward_infer(kind, xs, b1, out)
+        o = out.float().cpu().numpy()
+        assert o[0] == np.inf and o[1] == 0.0 and np.signbit(o[1]) and np.isnan(o[2]) and o[3] == 0.0
