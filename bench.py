@@ -390,7 +390,7 @@ def run_ours(args, w):
                 "d2h_bytes_per_step": 2 * n * es * len(kinds), "steps": e2e_steps,
                 "api": "nfad_host_step: pinned host x, grad_out in; y, grad_in out; copies and kernels pipelined by the library"},
         "gpu_launches": 2 * len(kinds) * args.steps,
-        "launch": ("CUDA graph of one buffer-rotation period (%d steps), last %d steps launched from the host, kernel by kernel, with events" % (period, period))
+        "launch": ("CUDA graph of one buffer-rotation period (%d steps); the last %d steps replayed from kernel-major graphs (one per kernel) between events" % (period, period))
                   if graph is not None else "every kernel launched from the host",
         "large_tensor_100663296": large,
         "clocks": sampler.summary(t_wall0, t_wall1, window) if sampler else None,
