@@ -12,6 +12,7 @@
 #include <stdio.h>
 #include <stdlib.h>
 #include <string.h>
+#include <unistd.h>
 
 #include <map>
 #include <mutex>
@@ -82,13 +83,23 @@ void open_api()
     Dl_info info;
     if (const char* env = getenv("NFAD_JIT_INCLUDE")) a.own_include = env;
     else if (dladdr(reinterpret_cast<void*>(&open_api), &info) && info.dli_fname) a.own_include = dir_of(info.dli_fname) + "/csrc";
-    // the toolkit's headers (cuda_bf16.h, cuda_fp16.h): beside the NVRTC that was loaded
-    if (const char* env = getenv("CUDA_HOME")) a.cuda_include = std::string(env) + "/include";
-    else if (dladdr(reinterpret_cast<void*>(a.create), &info) && info.dli_fname) {
+    // the toolkit's headers (cuda_bf16.h, cuda_fp16.h): the first of $CUDA_HOME/include, the include directory
+    // beside the NVRTC that was loaded, /usr/local/cuda/include that really holds them
+    std::vector<std::string> candidates;
+    if (const char* env = getenv("CUDA_HOME")) candidates.push_back(std::string(env) + "/include");
+    if (dladdr(reinterpret_cast<void*>(a.create), &info) && info.dli_fname) {
         char real[4096];
         std::string lib = realpath(info.dli_fname, real) ? std::string(real) : std::string(info.dli_fname);
-        a.cuda_include = dir_of(dir_of(lib)) + "/include";
-    } else a.cuda_include = "/usr/local/cuda/include";
+        candidates.push_back(dir_of(dir_of(lib)) + "/include");
+    }
+    candidates.push_back("/usr/local/cuda/include");
+    a.cuda_include = candidates.back();
+    for (const std::string& c : candidates) {
+        if (access((c + "/cuda_bf16.h").c_str(), R_OK) == 0) {
+            a.cuda_include = c;
+            break;
+        }
+    }
     a.ok = true;
 }
 
