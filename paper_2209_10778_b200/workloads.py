@@ -60,6 +60,9 @@ WORKLOADS = {
     "resnet50_stages": Workload("resnet50_stages", "f16", ("mish", "swish"),
                                 ((64, 64, 112, 112), (64, 256, 56, 56), (64, 512, 28, 28),
                                  (64, 1024, 14, 14), (64, 2048, 7, 7))),
+    # one feed-forward activation tensor of the 12-layer stack below (100.7M elements, 192 MiB: larger than L2),
+    # both GELU forms: the size class the bandwidth target is stated on
+    "gelu_ffn_100m": Workload("gelu_ffn_100m", "bf16", ("gelu_erf", "gelu_tanh"), ((64, 512, 3072),)),
     # 12 stacked GELU layers on [64, 512, 3072]
     "gelu_stack_12": Workload("gelu_stack_12", "bf16", ("gelu_erf",), ((64, 512, 3072),), layers=12),
 }

@@ -322,3 +322,50 @@ def test_bad_arguments_are_rejected():
         oracle.eval_point(7, 0.0)
     with pytest.raises(TypeError):
         oracle.forward("swish", "bf16", np.zeros(4, np.float32))
+
+
+# ----------------------------------------------------------------------------- stored 20-digit values
+
+def _closed_form_rows():
+    path = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden", "closed_forms.txt")
+    rows = []
+    with open(path) as fh:
+        for line in fh:
+            line = line.strip()
+            if line and not line.startswith("#"):
+                tag, kind, x, f, fp = line.split()
+                rows.append((tag, kind, float(x), float(f), float(fp)))
+    return rows
+
+
+def test_stored_closed_form_values():
+    """f and f' against the stored 50-digit evaluation of the literal definitions (Table I; x Phi(x)): the grid
+    into both tails, the stationary points of f', the sign change of f'.  No optional import: these pins hold on
+    any box.  f to 1e-13 relative; f' to 1e-13 of |h| + |x h'| (the size of the two terms it is the sum of)."""
+    rows = _closed_form_rows()
+    assert len(rows) == 54
+    assert {r[0] for r in rows} == {"table", "extremum", "root"}
+    for tag, kind, x, f_ref, fp_ref in rows:
+        f, fp, h, xh = oracle.eval_point(kind, x)
+        assert abs(f - f_ref) <= 1e-13 * abs(f_ref), (tag, kind, x, f, f_ref)
+        scale = abs(h) + abs(xh)
+        assert abs(fp - fp_ref) <= 1e-13 * scale, (tag, kind, x, fp, fp_ref)
+
+
+def test_stored_roots_and_extrema_have_their_closed_form_properties():
+    rows = _closed_form_rows()
+    ext = {(k, x > 0): (x, fp) for tag, k, x, f, fp in rows if tag == "extremum"}
+    # erf form: f'' = phi(x) (2 - x^2), so the stationary points of f' are +-sqrt(2)
+    assert abs(ext[("gelu_erf", True)][0] - math.sqrt(2.0)) < 1e-15 and abs(ext[("gelu_erf", False)][0] + math.sqrt(2.0)) < 1e-15
+    # the three kinds with h(x) + h(-x) = 1 have f'(x) + f'(-x) = 1 at their mirrored stationary points
+    for kind in ("gelu_erf", "gelu_tanh", "swish"):
+        (xp, fpp), (xn, fpn) = ext[(kind, True)], ext[(kind, False)]
+        assert abs(xp + xn) < 1e-15 and abs(fpp + fpn - 1.0) < 1e-15
+    # Swish: at the sign change of f', x s = x + 1
+    (xr, fr), = [(x, f) for tag, k, x, f, fp in rows if tag == "root" and k == "swish"]
+    assert abs(fr - (xr + 1.0)) < 1e-15
+    # a stationary point is a maximum (x > 0) or minimum (x < 0) of the oracle's f' too
+    for (kind, pos), (x, fp) in ext.items():
+        for dx in (-1e-3, 1e-3):
+            other = oracle.eval_point(kind, x + dx)[1]
+            assert (other < fp) if pos else (other > fp), (kind, x, dx)
