@@ -248,7 +248,7 @@ inline BiasPlan bias_plan(size_t rows, size_t cols, int sm_count)
     return p;
 }
 
-template <class S, bool kBf16>
+template <class S>
 __global__ void __launch_bounds__(kBiasMaxBlock, 4) bias_backward_kernel(const BiasBackwardArgs a)
 {
     constexpr int V = S::kVec;
@@ -286,7 +286,6 @@ __global__ void __launch_bounds__(kBiasMaxBlock, 4) bias_backward_kernel(const B
                     S::unpack(rd[u], vin[1]);
 #pragma unroll
                     for (int e = 0; e < V; ++e) vout[0][e] = __fmul_rn(vin[0][e], vin[1][e]);
-                    if constexpr (kBf16) BackwardOp<true>::template fixup<V>(vin, vout);
                     const uint4 packed = S::pack(vout[0]);
                     o4[(r + u) * a.row_packets + cp] = packed;
                     // the STORED values, widened again: what a reduction over the stored tensor would read
@@ -304,7 +303,7 @@ __global__ void __launch_bounds__(kBiasMaxBlock, 4) bias_backward_kernel(const B
 }
 
 // Any cols / alignment: a thread per column, the same chunks, rows added in the same order.
-template <class S, bool kBf16>
+template <class S>
 __global__ void __launch_bounds__(kBlock) bias_backward_scalar_kernel(const BiasBackwardArgs a)
 {
     using E = typename S::elem;
@@ -317,7 +316,7 @@ __global__ void __launch_bounds__(kBlock) bias_backward_scalar_kernel(const Bias
         const size_t i = r * a.cols + col;
         float in[2] = {S::load1(static_cast<const E*>(a.g) + i), S::load1(static_cast<const E*>(a.d) + i)};
         float out[1];
-        BackwardOp<kBf16>::apply_checked(in, out);
+        BackwardOp::apply(in, out);
         S::store1(static_cast<E*>(a.gin) + i, out[0]);
         acc = __fadd_rn(acc, S::load1(static_cast<const E*>(a.gin) + i));
     }
@@ -369,7 +368,7 @@ inline size_t bias_backward_scratch_bytes(size_t rows, size_t cols, int sm_count
     return p.chunks > 1 ? size_t(p.chunks) * cols * sizeof(float) : 0;
 }
 
-template <class S, bool kBf16>
+template <class S>
 cudaError_t launch_bias_backward(const void* g, const void* d, void* gin, float* grad_bias, void* scratch, size_t rows,
                                  size_t cols, cudaStream_t st)
 {
@@ -394,11 +393,11 @@ cudaError_t launch_bias_backward(const void* g, const void* d, void* gin, float*
     if (vec) {
         bias_launch_config(&cfg, attr, p.strips, p.block, st, true);
         cfg.gridDim.y = p.chunks;
-        e = cudaLaunchKernelEx(&cfg, bias_backward_kernel<S, kBf16>, a);
+        e = cudaLaunchKernelEx(&cfg, bias_backward_kernel<S>, a);
     } else {
         bias_launch_config(&cfg, attr, (cols + kBlock - 1) / kBlock, kBlock, st, false);
         cfg.gridDim.y = p.chunks;
-        e = cudaLaunchKernelEx(&cfg, bias_backward_scalar_kernel<S, kBf16>, a);
+        e = cudaLaunchKernelEx(&cfg, bias_backward_scalar_kernel<S>, a);
     }
     if (e != cudaSuccess || p.chunks == 1) return e;
     bias_launch_config(&cfg, attr, (cols + 31) / 32, 32 * kBiasGroups, st, true);

@@ -8,13 +8,13 @@
 
 namespace nfad {
 
-template <class S, class P, class K, bool kBf16>
+template <class S, class P, class K>
 cudaError_t dispatch_op(OpCode op, const void* const* in, void* const* out, size_t n, cudaStream_t st)
 {
     switch (op) {
     case kOpForward:      return launch_stream<S, ForwardTrainOp<K, P>>(in, out, n, st);
     case kOpForwardInfer: return launch_stream<S, ForwardInferOp<K, P>>(in, out, n, st);
-    case kOpBackward:     return launch_stream<S, BackwardOp<kBf16>>(in, out, n, st);
+    case kOpBackward:     return launch_stream<S, BackwardOp>(in, out, n, st);
     case kOpConvBackward: return launch_stream<S, ConvBackwardOp<K, P>>(in, out, n, st);
     case kOpRecompute1:   return launch_stream<S, RecomputePhase1Op<K, P>>(in, out, n, st);
     case kOpRecompute2:   return launch_stream<S, RecomputePhase2Op<K, P>>(in, out, n, st);
@@ -23,14 +23,14 @@ cudaError_t dispatch_op(OpCode op, const void* const* in, void* const* out, size
     return cudaErrorInvalidValue;
 }
 
-template <class S, class P, bool kBf16>
+template <class S, class P>
 cudaError_t dispatch_kind(OpCode op, int kind, const void* const* in, void* const* out, size_t n, cudaStream_t st)
 {
     switch (kind) {
-    case kGeluErf:  return dispatch_op<S, P, GeluErf, kBf16>(op, in, out, n, st);
-    case kGeluTanh: return dispatch_op<S, P, GeluTanh, kBf16>(op, in, out, n, st);
-    case kSwish:    return dispatch_op<S, P, Swish, kBf16>(op, in, out, n, st);
-    case kMish:     return dispatch_op<S, P, Mish, kBf16>(op, in, out, n, st);
+    case kGeluErf:  return dispatch_op<S, P, GeluErf>(op, in, out, n, st);
+    case kGeluTanh: return dispatch_op<S, P, GeluTanh>(op, in, out, n, st);
+    case kSwish:    return dispatch_op<S, P, Swish>(op, in, out, n, st);
+    case kMish:     return dispatch_op<S, P, Mish>(op, in, out, n, st);
     }
     return cudaErrorInvalidValue;
 }

@@ -9,8 +9,8 @@ namespace nfad {
 
 cudaError_t launch_16(OpCode op, int kind, int dtype, const void* const* in, void* const* out, size_t n, cudaStream_t st)
 {
-    if (dtype == kBF16) return dispatch_kind<StoreBF16, Fast, true>(op, kind, in, out, n, st);
-    if (dtype == kF16) return dispatch_kind<StoreF16, Fast, false>(op, kind, in, out, n, st);
+    if (dtype == kBF16) return dispatch_kind<StoreBF16, Fast>(op, kind, in, out, n, st);
+    if (dtype == kF16) return dispatch_kind<StoreF16, Fast>(op, kind, in, out, n, st);
     return cudaErrorInvalidValue;
 }
 

@@ -10,9 +10,9 @@ cudaError_t launch_bias_backward(int dtype, const void* g, const void* d, void* 
                                  size_t rows, size_t cols, cudaStream_t st)
 {
     switch (dtype) {
-    case kF32:  return launch_bias_backward<StoreF32, false>(g, d, gin, grad_bias, scratch, rows, cols, st);
-    case kBF16: return launch_bias_backward<StoreBF16, true>(g, d, gin, grad_bias, scratch, rows, cols, st);
-    case kF16:  return launch_bias_backward<StoreF16, false>(g, d, gin, grad_bias, scratch, rows, cols, st);
+    case kF32:  return launch_bias_backward<StoreF32>(g, d, gin, grad_bias, scratch, rows, cols, st);
+    case kBF16: return launch_bias_backward<StoreBF16>(g, d, gin, grad_bias, scratch, rows, cols, st);
+    case kF16:  return launch_bias_backward<StoreF16>(g, d, gin, grad_bias, scratch, rows, cols, st);
     }
     return cudaErrorInvalidValue;
 }

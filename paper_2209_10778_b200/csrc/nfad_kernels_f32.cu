@@ -68,7 +68,7 @@ cudaError_t launch_f32(OpCode op, int kind, const void* const* in, void* const* 
         }
         return cudaErrorInvalidValue;
     }
-    return dispatch_kind<StoreF32, Full, false>(op, kind, in, out, n, st);
+    return dispatch_kind<StoreF32, Full>(op, kind, in, out, n, st);
 }
 
 cudaError_t launch_bias_forward_f32(int kind, const void* x, const void* bias, void* y, void* d, size_t rows, size_t cols,

@@ -16,7 +16,6 @@ template <> struct IsFast<Fast> { static constexpr bool value = true; };
 #define NFAD_FWD16_UNROLL 5
 #endif
 template <class K, class P> struct ForwardTrainOp {
-    static constexpr bool kPacketFixup = false;
     static constexpr int kMinBlocks = 0;
     // 16-bit storage: 5 packets per thread measured 1-4 % faster than 4 (3 and 6 are slower)
     static constexpr int kUnroll = IsFast<P>::value ? NFAD_FWD16_UNROLL : 0;
@@ -32,7 +31,6 @@ template <class K, class P> struct ForwardTrainOp {
 
 // Forward, inference: x -> y.  Same chain; the tangent parts are dead code.
 template <class K, class P> struct ForwardInferOp {
-    static constexpr bool kPacketFixup = false;
     static constexpr int kMinBlocks = 0;
     static constexpr int kUnroll = 0;
     static constexpr int kIn = 1, kOut = 1;
@@ -44,57 +42,36 @@ template <class K, class P> struct ForwardInferOp {
 };
 
 // Backward of the nested layout (Eq. 4): grad_in = grad_out * f'(x), one multiply.
-// The fp32 product of two 16-bit values is exact unless it underflows; only bf16
-// shares fp32's exponent range, so only there can a product land below 2^-126,
-// where it is re-formed in fp64 and rounded straight to the bf16 subnormal grid
-// (multiples of 2^-133) to keep the result a single rounding of the true product.
-// That case is rare, so it is tested once per packet and handled out of line.
-static __device__ __noinline__ float bf16_tiny_product(float g, float d)
-{
-    const double kGrid = 6.2038417431289079e-25;   // 1.5 * 2^-81: its ulp is 2^-133
-    double pd = (double)g * (double)d;
-    pd = (pd + kGrid) - kGrid;
-    return (float)pd;
-}
-
+// One fp32 multiply followed by the store's rounding IS the single rounding of the exact
+// product, for every storage type:
+//   fp32: the multiply is that rounding.
+//   fp16: two 11-bit significands give a product of at most 22 bits inside fp32's normal
+//         range: exact, so the store's conversion is the only rounding.
+//   bf16: two 8-bit significands give M 2^e with M < 2^16.  At or above 2^-126 that is exact
+//         in fp32.  Below, fp32's grid is the multiples of 2^-149: a product whose leading bit
+//         is at 2^-134 or higher has its last bit at 2^-149 or higher and is exact again; one
+//         whose leading bit is lower is below 2^-134, half of bf16's smallest subnormal, and
+//         must become a zero of its sign: fp32 rounds it to at most 2^-134 (keeping the
+//         sign), which the store's round-to-nearest-even takes to that zero (2^-134 itself is
+//         the tie between 0 and 2^-133, and 0 is the even one).
+// So there is no double rounding to repair and no data-dependent path in this kernel.
 #ifndef NFAD_BWD_MIN_BLOCKS
 #define NFAD_BWD_MIN_BLOCKS 4
 #endif
 #ifndef NFAD_BWD_UNROLL
 #define NFAD_BWD_UNROLL 0
 #endif
-template <bool kBf16> struct BackwardOp {
+struct BackwardOp {
     static constexpr int kIn = 2, kOut = 1;
-    static constexpr bool kPacketFixup = kBf16;
     static constexpr int kMinBlocks = NFAD_BWD_MIN_BLOCKS;   // measured: 4 is 7 % faster than 5 for this load-and-multiply kernel
     static constexpr int kUnroll = NFAD_BWD_UNROLL;
     static __device__ __forceinline__ constexpr bool keep(int) { return true; }
-    static __device__ __forceinline__ void apply(const float (&in)[2], float (&out)[1]) { out[0] = in[0] * in[1]; }
-    // scalar path (edges): the same result, element by element
-    static __device__ __forceinline__ void apply_checked(const float (&in)[2], float (&out)[1])
-    {
-        float p = in[0] * in[1];
-        if (kBf16 && fabsf(p) <= 1.17549435e-38f) p = bf16_tiny_product(in[0], in[1]);
-        out[0] = p;
-    }
-    template <int V>
-    static __device__ __forceinline__ void fixup(const float (&vin)[2][V], float (&vout)[1][V])
-    {
-        bool tiny = false;
-#pragma unroll
-        for (int e = 0; e < V; ++e) tiny |= fabsf(vout[0][e]) <= 1.17549435e-38f;
-        if (tiny) {
-#pragma unroll                          // (a rolled loop would index the register arrays dynamically)
-            for (int e = 0; e < V; ++e)
-                if (fabsf(vout[0][e]) <= 1.17549435e-38f) vout[0][e] = bf16_tiny_product(vin[0][e], vin[1][e]);
-        }
-    }
+    static __device__ __forceinline__ void apply(const float (&in)[2], float (&out)[1]) { out[0] = __fmul_rn(in[0], in[1]); }
 };
 
 // Conventional layout: x is saved, and backward re-derives f'(x) with the full
 // transcendental chain before the multiply.
 template <class K, class P> struct ConvBackwardOp {
-    static constexpr bool kPacketFixup = false;
     static constexpr int kMinBlocks = 0;
     static constexpr int kUnroll = 0;
     static constexpr int kIn = 2, kOut = 1;
@@ -110,7 +87,6 @@ template <class K, class P> struct ConvBackwardOp {
 // per-operator backward rules need (the gate h = v1 of the Swish example), then
 // walks those rules: x' = g v1 + g v2 v1' with v2 = x (Eq. 2).
 template <class K, class P> struct RecomputePhase1Op {
-    static constexpr bool kPacketFixup = false;
     static constexpr int kMinBlocks = 0;
     static constexpr int kUnroll = 0;
     static constexpr int kIn = 1, kOut = 1;
@@ -153,7 +129,6 @@ template <> struct GateSlope<Mish> {
 };
 
 template <class K, class P> struct RecomputePhase2Op {
-    static constexpr bool kPacketFixup = false;
     static constexpr int kMinBlocks = 0;
     static constexpr int kUnroll = 0;
     static constexpr int kIn = 3, kOut = 1;            // grad_out, x, h
@@ -169,7 +144,6 @@ template <class K, class P> struct RecomputePhase2Op {
 // Traffic probe: moves bytes through the same streaming engine with no arithmetic to speak
 // of, to measure what a given read/write mix can reach on the device.
 template <int NIN, int NOUT> struct ProbeOp {
-    static constexpr bool kPacketFixup = false;
     static constexpr int kMinBlocks = 4;
     static constexpr int kUnroll = 0;
     static constexpr int kIn = NIN, kOut = NOUT;

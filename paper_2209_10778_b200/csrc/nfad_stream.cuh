@@ -40,10 +40,7 @@ template <int NIN, int NOUT> struct StreamArgs {
 //   static constexpr int kIn, kOut;  static constexpr bool keep(int out_slot);
 //   static __device__ void apply(const float (&in)[kIn], float (&out)[kOut]);
 //   static constexpr int kMinBlocks: resident CTAs per SM to leave room for (0: the storage type's default);
-//   static constexpr int kUnroll: packets per thread and tile (0: the default, 4);
-//   static constexpr bool kPacketFixup; if set, fixup(vin, vout) may patch a whole packet's
-//   results after apply (a rare case kept off the per-element path) and apply_checked is the
-//   one-element form that includes the patch.
+//   static constexpr int kUnroll: packets per thread and tile (0: the default, 4).
 template <class S, class Op>
 __device__ __forceinline__ void scalar_element(const StreamArgs<Op::kIn, Op::kOut>& a, size_t i)
 {
@@ -51,8 +48,7 @@ __device__ __forceinline__ void scalar_element(const StreamArgs<Op::kIn, Op::kOu
     float in[Op::kIn], out[Op::kOut];
 #pragma unroll
     for (int k = 0; k < Op::kIn; ++k) in[k] = S::load1(static_cast<const E*>(a.in[k]) + i);
-    if constexpr (Op::kPacketFixup) Op::apply_checked(in, out);
-    else Op::apply(in, out);
+    Op::apply(in, out);
 #pragma unroll
     for (int k = 0; k < Op::kOut; ++k) S::store1(static_cast<E*>(a.out[k]) + i, out[k]);
 }
@@ -75,7 +71,6 @@ __device__ __forceinline__ void packet_compute_store(const StreamArgs<Op::kIn, O
 #pragma unroll
         for (int k = 0; k < Op::kOut; ++k) vout[k][e] = out[k];
     }
-    if constexpr (Op::kPacketFixup) Op::template fixup<V>(vin, vout);
     const size_t byte_off = a.head * sizeof(typename S::elem);
 #pragma unroll
     for (int k = 0; k < Op::kOut; ++k) {

@@ -68,7 +68,6 @@ template <class K> __device__ __forceinline__ ActOut evaluate_strict(float x)
 }
 
 template <class K> struct ForwardStrictOp {
-    static constexpr bool kPacketFixup = false;
     static constexpr int kMinBlocks = 3;
     static constexpr int kUnroll = 2;
     static constexpr int kIn = 1, kOut = 2;

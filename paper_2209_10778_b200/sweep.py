@@ -48,24 +48,28 @@ def _peak():
         return 6650.0, "fallback"
 
 
-def _make_sets(n, dtype, n_tensors, dev, std=1.0):
+def _make_sets(n, dtype, n_tensors, dev, std=1.0, dist="normal"):
+    """dist: how x is drawn -- "normal" (N(0, std^2)), "uniform20" (U(-20, 20)), "mix" (the stress mix with
+    magnitudes up to 80), or "tiny" (x ~ N(0,1), and grad_out ~ N(0, (1e-38)^2) -- 1e-6 for fp16 --
+    so that most backward products land in the storage type's subnormal range)."""
     es = 4 if dtype == "f32" else 2
     per_set = n_tensors * n * es
     n_sets = 1 if n * es > L2_BYTES else max(2, -(-4 * L2_BYTES // per_set))
     n_sets = min(n_sets, 256)
     sets = []
     for i in range(n_sets):
-        x = W.normal(n, dtype, 10 + i, std, dev)
-        g = W.normal(n, dtype, 500 + i, 1.0, dev)
+        x = W.normal(n, dtype, 10 + i, std, dev) if dist in ("normal", "tiny") else W.draw(dist, n, dtype, 10 + i, dev)
+        g = W.normal(n, dtype, 500 + i, (1e-6 if dtype == "f16" else 1e-38) if dist == "tiny" else 1.0, dev)
         s = {"x": x, "g": g, "y": torch.empty_like(x), "d": torch.empty_like(x), "gin": torch.empty_like(x)}
         sets.append(s)
     return sets
 
 
-def time_case(kind: str, dtype: str, op: str, n: int, reps: int = 20, dev="cuda", std=1.0, cols: int = 3072, repeats: int = 10):
+def time_case(kind: str, dtype: str, op: str, n: int, reps: int = 20, dev="cuda", std=1.0, cols: int = 3072, repeats: int = 10,
+              dist: str = "normal"):
     """cols: row length for the bias-fused calls (n must be a multiple of it)."""
     es = 4 if dtype == "f32" else 2
-    sets = _make_sets(n, dtype, 5, dev, std)
+    sets = _make_sets(n, dtype, 5, dev, std, dist)
     if op.startswith("bias_"):
         rows = n // cols
         bias = W.normal(cols, dtype, 3, 0.5, dev)
@@ -124,7 +128,7 @@ def time_case(kind: str, dtype: str, op: str, n: int, reps: int = 20, dev="cuda"
     return {"kind": kind, "dtype": dtype, "op": op, "n": n, "ms": ms, "elements_per_s": n / (ms / 1e3),
             "algorithmic_bytes": algo, "GBps": gbs, "frac_of_peak": gbs / peak, "peak_GBps": peak, "peak_source": src,
             "frac_of_nominal_8000": gbs / 8000.0, "buffer_sets": len(sets), "launches_per_burst": per_burst, "bursts": repeats,
-            "ms_min": min(samples), "ms_max": max(samples), "x_std": std,
+            "ms_min": min(samples), "ms_max": max(samples), "x_std": std, "dist": dist,
             "inputs": {"generator": "torch.Generator(device).manual_seed", "x_seed": "10 + set index", "g_seed": "500 + set index",
                        "torch": torch.__version__}}
 
@@ -362,9 +366,11 @@ def main(argv=None):
     ap.add_argument("--n", type=int, default=100663296)
     ap.add_argument("--kinds", default="gelu_erf,gelu_tanh,swish,mish")
     ap.add_argument("--dtypes", default="bf16")
+    ap.add_argument("--dists", default="normal", help="input distributions: normal, uniform20, mix, tiny (backward: products in fp32's subnormal range)")
     ap.add_argument("--ops", default="forward,backward")
     ap.add_argument("--reps", type=int, default=20)
     ap.add_argument("--max-log2", type=int, default=30)
+    ap.add_argument("--min-log2", type=int, default=16)
     ap.add_argument("--repeats", type=int, default=10, help="bursts per case (1 under a profiler: the burst is then `reps` launches)")
     args = ap.parse_args(argv)
     if not torch.cuda.is_available():
@@ -383,16 +389,18 @@ def main(argv=None):
 
 def _run_config(args):
     kinds, dtypes, ops = args.kinds.split(","), args.dtypes.split(","), args.ops.split(",")
+    dists = args.dists.split(",")
     if args.config == "sizes":
         for n in W.SWEEP_SIZES:
-            if n > (1 << args.max_log2):
+            if n > (1 << args.max_log2) or n < (1 << args.min_log2):
                 continue
             for dtype in dtypes:
-                for kind in kinds:
-                    for op in ops:
-                        reps = max(3, min(args.reps, (1 << 28) // n + 3))
-                        print(json.dumps(time_case(kind, dtype, op, n, reps)), flush=True)
-                        torch.cuda.empty_cache()
+                for dist in dists:
+                    for kind in kinds:
+                        for op in ops:
+                            reps = max(3, min(args.reps, (1 << 28) // n + 3))
+                            print(json.dumps(time_case(kind, dtype, op, n, reps, dist=dist)), flush=True)
+                            torch.cuda.empty_cache()
     elif args.config == "resnet50":
         w = W.WORKLOADS["resnet50_stages"]
         for si, shape in enumerate(w.shapes):
@@ -426,10 +434,12 @@ def _run_config(args):
             print(json.dumps(r), flush=True)
     else:
         for dtype in dtypes:
-            for kind in kinds:
-                for op in ops:
-                    print(json.dumps(time_case(kind, dtype, op, args.n, args.reps, cols=args.cols, repeats=args.repeats)), flush=True)
-                    torch.cuda.empty_cache()
+            for dist in dists:
+                for kind in kinds:
+                    for op in ops:
+                        print(json.dumps(time_case(kind, dtype, op, args.n, args.reps, cols=args.cols, repeats=args.repeats,
+                                                   dist=dist)), flush=True)
+                        torch.cuda.empty_cache()
 
 
 if __name__ == "__main__":

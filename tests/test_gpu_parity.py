@@ -130,3 +130,20 @@ def test_non_finite_inputs(kind, dtype):
         assert y[i] == xf[i] and d[i] == 1.0
     for i in (4, 6):
         assert y[i] == 0.0 and d[i] == 0.0
+
+
+def test_backward_bf16_products_that_round_to_signed_zero_or_the_smallest_subnormal():
+    # products between 2^-150 and 2^-130: fp32 cannot hold them exactly, the bf16 result is +-0 or a few subnormals;
+    # the bits (sign of a zero included) must be those of ONE rounding of the exact product
+    rng = np.random.default_rng(11)
+    n = 200000
+    a = 2.0 ** rng.uniform(-80, -60, n) * rng.choice([-1, 1], n)
+    b = 2.0 ** rng.uniform(-72, -66, n) * rng.choice([-1, 1], n)
+    g_raw, d_raw = oracle.round_to("bf16", a), oracle.round_to("bf16", b)
+    g = W.from_raw_numpy(g_raw, "bf16", DEV)
+    d = W.from_raw_numpy(d_raw, "bf16", DEV)
+    gin = parity.gpu_backward("gelu_erf", g, d)
+    torch.cuda.synchronize()
+    got = W.raw_numpy(gin)
+    parity.check_backward("bf16", g_raw, d_raw, got)
+    assert (got == 0x8000).any() and (got == 0x0000).any() and ((got & 0x7FFF) == 1).any()   # the cases are really there

@@ -62,9 +62,11 @@ def is_nan16(bits: np.ndarray, dtype: str) -> np.ndarray:
 
 
 def same_bits_or_both_nan(a: np.ndarray, b: np.ndarray, dtype: str) -> np.ndarray:
-    """Bit equality, with +0 == -0 and NaN == NaN (backward parity)."""
+    """Equality of the raw bit patterns (so +0 and -0 differ: a single rounding of the exact product fixes the
+    sign of a zero too), any NaN equal to any NaN (backward parity)."""
     if dtype == "f32":
         a32 = np.ascontiguousarray(a, np.float32)
         b32 = np.ascontiguousarray(b, np.float32)
-        return (ord32(a32) == ord32(b32)) | (np.isnan(a32) & np.isnan(b32))
-    return (ord16(a) == ord16(b)) | (is_nan16(a, dtype) & is_nan16(b, dtype))
+        return (a32.view(np.uint32) == b32.view(np.uint32)) | (np.isnan(a32) & np.isnan(b32))
+    a16, b16 = np.asarray(a).view(np.uint16), np.asarray(b).view(np.uint16)
+    return (a16 == b16) | (is_nan16(a, dtype) & is_nan16(b, dtype))
