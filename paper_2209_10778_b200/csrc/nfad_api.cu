@@ -118,6 +118,17 @@ int check_shape(size_t rows, size_t cols, size_t* n)
 
 namespace nfad {
 void note_cuda_error(cudaError_t e) { g_last_cuda_error = static_cast<int>(e); }
+
+unsigned edge_grid_blocks(size_t n, unsigned block)
+{
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
+        sms = 128;
+    size_t need = (n + block - 1) / block;
+    size_t cap = size_t(sms) * 32;
+    if (need == 0) need = 1;
+    return (unsigned)(need < cap ? need : cap);
+}
 }  // namespace nfad
 
 extern "C" {

@@ -46,6 +46,14 @@ NFAD_DEV float lg2_approx(float a)
     return r;
 }
 
+// min(a, hi) that returns NaN for a NaN.
+NFAD_DEV float min_nan(float a, float hi)
+{
+    float r;
+    asm("min.NaN.f32 %0, %1, %2;" : "=f"(r) : "f"(a), "f"(hi));
+    return r;
+}
+
 // max(a, lo) that returns NaN for a NaN.
 NFAD_DEV float max_nan(float a, float lo)
 {
@@ -61,6 +69,21 @@ NFAD_DEV float rcp_approx(float a)
     asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(a));
     return r;
 }
+
+// 1/a for a normal double a: MUFU.RCP64H, an estimate from the upper word good to about 20 bits.
+NFAD_DEV double rcp64_approx(double a)
+{
+    double r;
+    asm("rcp.approx.ftz.f64 %0, %1;" : "=d"(r) : "d"(a));
+    return r;
+}
+
+// the two 32-bit words of a double, and a double from them
+NFAD_DEV int double_hi(double a) { return __double2hiint(a); }
+NFAD_DEV int double_lo(double a) { return __double2loint(a); }
+NFAD_DEV double double_from(int hi, int lo) { return __hiloint2double(hi, lo); }
+// double -> float, round to nearest even (subnormal results included)
+NFAD_DEV float to_float(double a) { return __double2float_rn(a); }
 
 NFAD_DEV int float_as_int(float a) { return __float_as_int(a); }
 NFAD_DEV float int_as_float(int a) { return __int_as_float(a); }

@@ -49,6 +49,10 @@ std::string seq_generate_source(const SeqProgramHost& p, int dtype, int m);   //
 cudaError_t launch_seq_backward(int dtype, const void* const* g, const void* const* d, int m, void* gin, size_t n, cudaStream_t st);
 cudaError_t launch_ew(int op, int backward, float c, int dtype, const void* const* in, void* const* out, size_t n, cudaStream_t st);
 
+// CTAs for a launch that takes n elements one by one with a grid-stride loop: enough to fill the current device
+// (32 CTAs of `block` threads per SM at most), never more than the elements need.
+unsigned edge_grid_blocks(size_t n, unsigned block);
+
 // Records the cudaError_t behind an NFAD_E_CUDA of the calling thread (what nfad_last_cuda_error() returns).
 void note_cuda_error(cudaError_t e);
 

@@ -111,29 +111,34 @@ const char* kOpExpr[] = {
 
 std::string generate(const SeqProgramHost& p, int m, const char* store)
 {
+    // fp32 tensors run under the double-precision policy, 16-bit tensors under the fp32 one (as the interpreter does)
+    const bool wide = strcmp(store, "StoreF32") == 0;
+    const char* pol = wide ? "Wide" : "Fast";
     char buf[512];
     std::string s = "#include \"nfad_jit_kernel.cuh\"\nnamespace nfad {\n";
     snprintf(buf, sizeof buf, "template <> __device__ __forceinline__ void jit_element<%d>(float x, float (&yv)[%d], float (&yt)[%d])\n{\n", m, m, m);
     s += buf;
-    s += "    const Dual<Fast> v_src{x, 1.0f};\n";
+    snprintf(buf, sizeof buf, wide ? "    const Dual<%s> v_src{double(x), 1.0};\n" : "    const Dual<%s> v_src{x, 1.0f};\n", pol);
+    s += buf;
     std::string reg[12];
     reg[0] = "v_src";
     for (int i = 0; i < p.n_ops; ++i) {
         const std::string a = reg[p.a[i]], b = reg[p.b[i]];
         if (p.op[i] == 12) {                       // OUT
-            snprintf(buf, sizeof buf, "    yv[%d] = %s.v; yt[%d] = %s.t;\n", p.dst[i], a.c_str(), p.dst[i], a.c_str());
+            snprintf(buf, sizeof buf, "    yv[%d] = dual_value(%s); yt[%d] = dual_tangent(%s);\n", p.dst[i], a.c_str(), p.dst[i], a.c_str());
             s += buf;
             continue;
         }
         unsigned bits;
         float c = p.c[i];
         memcpy(&bits, &c, 4);
-        char expr[256];
-        if (p.op[i] == 2) snprintf(expr, sizeof expr, "Dual<Fast>{__int_as_float(0x%08x) * %s.v, __int_as_float(0x%08x) * %s.t}", bits, a.c_str(), bits, a.c_str());
-        else if (p.op[i] == 3) snprintf(expr, sizeof expr, "dual_add_const(__int_as_float(0x%08x), %s)", bits, a.c_str());
+        char cst[64], expr[256];
+        snprintf(cst, sizeof cst, wide ? "double(__int_as_float(0x%08x))" : "__int_as_float(0x%08x)", bits);
+        if (p.op[i] == 2) snprintf(expr, sizeof expr, "dual_scale(%s, %s)", cst, a.c_str());
+        else if (p.op[i] == 3) snprintf(expr, sizeof expr, "dual_add_const(%s, %s)", cst, a.c_str());
         else if (p.op[i] < 2) snprintf(expr, sizeof expr, kOpExpr[p.op[i]], a.c_str(), b.c_str());
         else snprintf(expr, sizeof expr, kOpExpr[p.op[i]], a.c_str());
-        snprintf(buf, sizeof buf, "    const Dual<Fast> v%d = %s;\n", i, expr);
+        snprintf(buf, sizeof buf, "    const Dual<%s> v%d = %s;\n", pol, i, expr);
         s += buf;
         snprintf(buf, sizeof buf, "v%d", i);
         reg[p.dst[i]] = buf;
@@ -250,6 +255,7 @@ cudaError_t launch_seq_forward_compiled(const SeqProgramHost& p, int dtype, cons
     }
     const size_t tile = size_t(256) * kJitUnroll;
     size_t blocks = (a.packets + tile - 1) / tile;
+    if (!congruent) blocks = edge_grid_blocks(n, 256);      // every element goes through the element-wise path: fill the device
     if (blocks == 0) blocks = 1;
     if (blocks > 0x7fffffffull) blocks = 0x7fffffffull;
     void* params[1] = {&a};

@@ -70,10 +70,12 @@ template <class S, int M> __device__ __forceinline__ void jit_forward(const JitA
             }
         }
     }
-    if (blockIdx.x == 0) {                         // ragged ends, one element at a time, the same code
+    {   // outside the packet grid, one element at a time with the same code, spread over the whole grid: a few at the
+        // ragged ends, or all n when the tensors share no offset modulo 16 bytes (head = n, packets = 0)
         const unsigned long long tail_begin = a.head + a.packets * V;
         const unsigned long long n_edge = a.head + (a.n - tail_begin);
-        for (unsigned long long j = threadIdx.x; j < n_edge; j += blockDim.x) {
+        for (unsigned long long j = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x; j < n_edge;
+             j += (unsigned long long)gridDim.x * blockDim.x) {
             const unsigned long long i = j < a.head ? j : tail_begin + (j - a.head);
             float v[M], t[M];
             jit_element<M>(S::load1(static_cast<const E*>(a.x) + i), v, t);

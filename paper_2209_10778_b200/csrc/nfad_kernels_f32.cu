@@ -1,6 +1,6 @@
-// fp32-storage kernels (Full precision policy).  Build with -fmad=false: the
-// compensated arithmetic in nfad_numerics.cuh names every fused multiply-add
-// explicitly and must not have others introduced by contraction.
+// fp32-storage kernels (Wide policy: the chains run in double precision and name every fused
+// multiply-add explicitly).  Built with -fmad=false so that the few fp32 operations in this
+// unit (the bias addition z = x + b, the comparators' rules) are rounded as written.
 #include "nfad_bias.cuh"
 #include "nfad_dispatch.cuh"
 #include "nfad_strict.cuh"
@@ -68,17 +68,17 @@ cudaError_t launch_f32(OpCode op, int kind, const void* const* in, void* const* 
         }
         return cudaErrorInvalidValue;
     }
-    return dispatch_kind<StoreF32, Full>(op, kind, in, out, n, st);
+    return dispatch_kind<StoreF32, Wide>(op, kind, in, out, n, st);
 }
 
 cudaError_t launch_bias_forward_f32(int kind, const void* x, const void* bias, void* y, void* d, size_t rows, size_t cols,
                                     cudaStream_t st)
 {
     switch (kind) {
-    case kGeluErf:  return launch_bias_forward<StoreF32, GeluErf, Full>(x, bias, y, d, rows, cols, st);
-    case kGeluTanh: return launch_bias_forward<StoreF32, GeluTanh, Full>(x, bias, y, d, rows, cols, st);
-    case kSwish:    return launch_bias_forward<StoreF32, Swish, Full>(x, bias, y, d, rows, cols, st);
-    case kMish:     return launch_bias_forward<StoreF32, Mish, Full>(x, bias, y, d, rows, cols, st);
+    case kGeluErf:  return launch_bias_forward<StoreF32, GeluErf, Wide>(x, bias, y, d, rows, cols, st);
+    case kGeluTanh: return launch_bias_forward<StoreF32, GeluTanh, Wide>(x, bias, y, d, rows, cols, st);
+    case kSwish:    return launch_bias_forward<StoreF32, Swish, Wide>(x, bias, y, d, rows, cols, st);
+    case kMish:     return launch_bias_forward<StoreF32, Mish, Wide>(x, bias, y, d, rows, cols, st);
     }
     return cudaErrorInvalidValue;
 }

@@ -1,5 +1,5 @@
-// Run-time FAD sequences and single-operator kernels (Fast policy arithmetic for every
-// storage type: plain fp32).  Built with contraction on, like the 16-bit kernels.
+// Run-time FAD sequences and single-operator kernels: the fp32 primitives for 16-bit storage, the
+// double-precision ones for fp32 storage.  Built with contraction on, like the 16-bit kernels.
 #include "nfad_internal.h"
 #include "nfad_seq.cuh"
 
@@ -7,13 +7,32 @@ namespace nfad {
 
 namespace {
 
-template <class T> bool aligned16(const T* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
-
 unsigned grid_for(size_t items)
 {
     size_t blocks = (items + kBlock - 1) / kBlock;
     if (blocks == 0) blocks = 1;
     return (unsigned)(blocks < size_t(0x7fffffff) ? blocks : size_t(0x7fffffff));
+}
+
+// Where the packet grid of a call starts: if every tensor has the same offset modulo 16 bytes, `head` elements
+// come before the first common 16-byte boundary and whole packets follow; if not, no packet grid exists and every
+// element goes through the kernels' element-wise path (head = n), which then gets a grid that fills the device.
+struct PacketSplit { size_t head, packets; bool congruent; };
+
+PacketSplit packet_split(const void* const* ptrs, int count, size_t n, size_t esz)
+{
+    uintptr_t mis = 0;
+    bool congruent = true, first = true;
+    for (int k = 0; k < count; ++k) {
+        if (!ptrs[k]) continue;
+        uintptr_t m = reinterpret_cast<uintptr_t>(ptrs[k]) & 15u;
+        if (first) { mis = m; first = false; }
+        congruent = congruent && m == mis;
+    }
+    if (!congruent || (mis % esz) != 0) return {n, 0, false};
+    size_t head = ((16u - mis) & 15u) / esz;
+    if (head > n) head = n;
+    return {head, (n - head) / (16 / esz), true};
 }
 
 template <class K, class A> cudaError_t launch_pdl(K kernel, unsigned grid, cudaStream_t st, const A& args)
@@ -35,44 +54,41 @@ cudaError_t seq_forward_t(const SeqProgram& prog, const void* x, void* const* y,
 {
     SeqForwardArgs a;
     a.x = x;
-    uintptr_t mis = reinterpret_cast<uintptr_t>(x) & 15u;
-    bool congruent = true;
+    const void* ptrs[1 + 2 * kSeqMaxOut] = {x};
     for (int k = 0; k < kSeqMaxOut; ++k) {
         a.y[k] = k < m ? y[k] : nullptr;
         a.d[k] = k < m ? d[k] : nullptr;
-        if (k < m) congruent = congruent && ((reinterpret_cast<uintptr_t>(y[k]) & 15u) == mis) && ((reinterpret_cast<uintptr_t>(d[k]) & 15u) == mis);
+        ptrs[1 + 2 * k] = a.y[k];
+        ptrs[2 + 2 * k] = a.d[k];
     }
     a.m = m;
     a.n = n;
-    constexpr size_t esz = sizeof(typename S::elem);
-    if (congruent) {
-        size_t head = ((16u - mis) & 15u) / esz;
-        a.head = head > n ? n : head;
-        a.packets = (n - a.head) / S::kVec;
-    } else {                       // no common packet grid: everything through the element-wise edge path
-        a.head = n;
-        a.packets = 0;
-    }
+    const PacketSplit sp = packet_split(ptrs, 1 + 2 * kSeqMaxOut, n, sizeof(typename S::elem));
+    a.head = sp.head;
+    a.packets = sp.packets;
     a.prog = prog;
-    return launch_pdl(seq_forward_kernel<S>, grid_for(a.packets), st, a);
+    return launch_pdl(seq_forward_kernel<S>, sp.congruent ? grid_for(a.packets) : edge_grid_blocks(n, kBlock), st, a);
 }
 
 template <class S>
 cudaError_t seq_backward_t(const void* const* g, const void* const* d, int m, void* gin, size_t n, cudaStream_t st)
 {
     SeqBackwardArgs a;
-    bool al = aligned16(gin);
+    const void* ptrs[1 + 2 * kSeqMaxOut] = {gin};
     for (int k = 0; k < kSeqMaxOut; ++k) {
         a.g[k] = k < m ? g[k] : nullptr;
         a.d[k] = k < m ? d[k] : nullptr;
-        if (k < m) al = al && aligned16(g[k]) && aligned16(d[k]);
+        ptrs[1 + 2 * k] = a.g[k];
+        ptrs[2 + 2 * k] = a.d[k];
     }
     a.gin = gin;
     a.m = m;
     a.n = n;
-    a.packets = al ? n / S::kVec : 0;
+    const PacketSplit sp = packet_split(ptrs, 1 + 2 * kSeqMaxOut, n, sizeof(typename S::elem));
+    a.head = sp.head;
+    a.packets = sp.packets;
     const int u = seq_bwd_unroll(m);
-    const unsigned grid = grid_for(al ? (a.packets + u - 1) / u : 0);
+    const unsigned grid = sp.congruent ? grid_for((a.packets + u - 1) / u) : edge_grid_blocks(n, kBlock);
     switch (m) {
     case 1: return launch_pdl(seq_backward_kernel<S, 1>, grid, st, a);
     case 2: return launch_pdl(seq_backward_kernel<S, 2>, grid, st, a);
@@ -85,15 +101,17 @@ template <class S>
 cudaError_t ew_t(int op, int backward, float c, const void* const* in, void* const* out, size_t n, cudaStream_t st)
 {
     EwArgs a;
-    bool al = true;
-    for (int k = 0; k < 3; ++k) { a.in[k] = in[k]; if (in[k]) al = al && aligned16(in[k]); }
-    for (int k = 0; k < 2; ++k) { a.out[k] = out[k]; if (out[k]) al = al && aligned16(out[k]); }
+    const void* ptrs[5];
+    for (int k = 0; k < 3; ++k) { a.in[k] = in[k]; ptrs[k] = in[k]; }
+    for (int k = 0; k < 2; ++k) { a.out[k] = out[k]; ptrs[3 + k] = out[k]; }
     a.op = op;
     a.backward = backward;
     a.c = c;
     a.n = n;
-    a.packets = al ? n / S::kVec : 0;
-    const unsigned grid = grid_for(al ? (a.packets + kEwUnroll - 1) / kEwUnroll : 0);
+    const PacketSplit sp = packet_split(ptrs, 5, n, sizeof(typename S::elem));
+    a.head = sp.head;
+    a.packets = sp.packets;
+    const unsigned grid = sp.congruent ? grid_for((a.packets + kEwUnroll - 1) / kEwUnroll) : edge_grid_blocks(n, kBlock);
 #define NFAD_EW_CASE(OPC) \
     case OPC: return backward ? launch_pdl(ew_kernel<S, OPC, true>, grid, st, a) : launch_pdl(ew_kernel<S, OPC, false>, grid, st, a);
     switch (op) {

@@ -72,7 +72,9 @@ struct BackwardOp {
 // Conventional layout: x is saved, and backward re-derives f'(x) with the full
 // transcendental chain before the multiply.
 template <class K, class P> struct ConvBackwardOp {
-    static constexpr int kMinBlocks = 0;
+    // two input streams of four packets each are 32 registers before any arithmetic: room for 64 (four resident CTAs),
+    // or the chain's temporaries spill
+    static constexpr int kMinBlocks = 4;
     static constexpr int kUnroll = 0;
     static constexpr int kIn = 2, kOut = 1;
     static __device__ __forceinline__ constexpr bool keep(int) { return true; }
@@ -129,8 +131,9 @@ template <> struct GateSlope<Mish> {
 };
 
 template <class K, class P> struct RecomputePhase2Op {
-    static constexpr int kMinBlocks = 0;
-    static constexpr int kUnroll = 0;
+    // three input streams: three packets each and 64 registers (see ConvBackwardOp)
+    static constexpr int kMinBlocks = 4;
+    static constexpr int kUnroll = 3;
     static constexpr int kIn = 3, kOut = 1;            // grad_out, x, h
     static __device__ __forceinline__ constexpr bool keep(int) { return true; }
     static __device__ __forceinline__ void apply(const float (&in)[3], float (&out)[1])

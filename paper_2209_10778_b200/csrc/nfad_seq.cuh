@@ -32,14 +32,23 @@ enum SeqOpcode {
 struct SeqOp { int op, a, b, dst; float c; };
 struct SeqProgram { int n_ops; SeqOp ops[kSeqMaxOps]; };
 
-// One primitive on duals (Fast policy: plain fp32).
-__device__ __forceinline__ Dual<Fast> seq_apply(const SeqOp& o, const Dual<Fast>& a, const Dual<Fast>& b)
+// The policy a storage type's sequences run under, and that policy's scalar: fp32 tensors get the double-precision
+// primitives (results within an fp32 rounding or two of the exact ones), 16-bit tensors the fp32 ones.
+template <class S> struct SeqPolicy { using type = Fast; };
+template <> struct SeqPolicy<StoreF32> { using type = Wide; };
+template <class P> struct ScalarOf { using type = float; };
+template <> struct ScalarOf<Wide> { using type = double; };
+
+// One primitive on duals.
+template <class P>
+__device__ __forceinline__ Dual<P> seq_apply(const SeqOp& o, const Dual<P>& a, const Dual<P>& b)
 {
+    using T = typename ScalarOf<P>::type;
     switch (o.op) {
     case kSeqAdd: return dual_add(a, b);
     case kSeqMul: return dual_mul(a, b);
-    case kSeqScale: return Dual<Fast>{o.c * a.v, o.c * a.t};
-    case kSeqAddConst: return dual_add_const(o.c, a);
+    case kSeqScale: return dual_scale(T(o.c), a);
+    case kSeqAddConst: return dual_add_const(T(o.c), a);
     case kSeqExp: return dual_exp(a);
     case kSeqLog1p: return dual_log1p(a);
     case kSeqTanh: return dual_tanh(a);
@@ -53,32 +62,37 @@ __device__ __forceinline__ Dual<Fast> seq_apply(const SeqOp& o, const Dual<Fast>
 }
 
 // Interprets the program for V elements, kSeqGroup at a time: the register file is indexed at
-// run time and so lives in local memory, and kSeqRegs x 2 x kSeqGroup floats per thread is what
+// run time and so lives in local memory, and kSeqRegs x 2 x kSeqGroup scalars per thread is what
 // has to stay inside L1 for every resident thread.
 #ifndef NFAD_SEQ_GROUP
 #define NFAD_SEQ_GROUP 2
 #endif
 constexpr int kSeqGroup = NFAD_SEQ_GROUP;
 
-template <int V>
+template <class P, int V>
 __device__ __forceinline__ void seq_run(const SeqProgram& prog, const float (&x)[V], float (&yv)[kSeqMaxOut][V],
                                         float (&yt)[kSeqMaxOut][V])
 {
+    using T = typename ScalarOf<P>::type;
     constexpr int G = V < kSeqGroup ? V : kSeqGroup;
 #pragma unroll
     for (int e0 = 0; e0 < V; e0 += G) {
-        float rv[kSeqRegs][G], rt[kSeqRegs][G];
+        T rv[kSeqRegs][G], rt[kSeqRegs][G];
 #pragma unroll
-        for (int e = 0; e < G; ++e) { rv[0][e] = x[e0 + e]; rt[0][e] = 1.0f; }
+        for (int e = 0; e < G; ++e) { rv[0][e] = T(x[e0 + e]); rt[0][e] = T(1); }
         for (int i = 0; i < prog.n_ops; ++i) {
             const SeqOp o = prog.ops[i];
             if (o.op == kSeqOut) {
 #pragma unroll
-                for (int e = 0; e < G; ++e) { yv[o.dst][e0 + e] = rv[o.a][e]; yt[o.dst][e0 + e] = rt[o.a][e]; }
+                for (int e = 0; e < G; ++e) {
+                    const Dual<P> r{rv[o.a][e], rt[o.a][e]};
+                    yv[o.dst][e0 + e] = dual_value(r);
+                    yt[o.dst][e0 + e] = dual_tangent(r);
+                }
             } else {
 #pragma unroll
                 for (int e = 0; e < G; ++e) {
-                    Dual<Fast> r = seq_apply(o, Dual<Fast>{rv[o.a][e], rt[o.a][e]}, Dual<Fast>{rv[o.b][e], rt[o.b][e]});
+                    Dual<P> r = seq_apply<P>(o, Dual<P>{rv[o.a][e], rt[o.a][e]}, Dual<P>{rv[o.b][e], rt[o.b][e]});
                     rv[o.dst][e] = r.v;
                     rt[o.dst][e] = r.t;
                 }
@@ -108,20 +122,22 @@ __global__ void __launch_bounds__(kBlock) seq_forward_kernel(const SeqForwardArg
         uint4 raw = load_packet(reinterpret_cast<const uint4*>(static_cast<const char*>(a.x) + byte_off) + pk);
         float xv[V], yv[kSeqMaxOut][V], yt[kSeqMaxOut][V];
         S::unpack(raw, xv);
-        seq_run<V>(a.prog, xv, yv, yt);
+        seq_run<typename SeqPolicy<S>::type, V>(a.prog, xv, yv, yt);
         for (int k = 0; k < a.m; ++k) {
             *(reinterpret_cast<uint4*>(static_cast<char*>(a.y[k]) + byte_off) + pk) = S::pack(yv[k]);
             __stcs(reinterpret_cast<uint4*>(static_cast<char*>(a.d[k]) + byte_off) + pk, S::pack(yt[k]));
         }
     }
-    if (blockIdx.x == 0) {
+    // elements outside the packet grid, one by one, spread over the whole grid: a few at the ragged ends when the tensors
+    // share one offset modulo 16 bytes, all n of them when they do not (head = n, packets = 0)
+    {
         const size_t tail_begin = a.head + a.packets * V;
         const size_t n_edge = a.head + (a.n - tail_begin);
-        for (size_t j = threadIdx.x; j < n_edge; j += kBlock) {
+        for (size_t j = size_t(blockIdx.x) * kBlock + threadIdx.x; j < n_edge; j += size_t(gridDim.x) * kBlock) {
             const size_t i = j < a.head ? j : tail_begin + (j - a.head);
             float xv[1] = {S::load1(static_cast<const E*>(a.x) + i)};
             float yv[kSeqMaxOut][1], yt[kSeqMaxOut][1];
-            seq_run<1>(a.prog, xv, yv, yt);
+            seq_run<typename SeqPolicy<S>::type, 1>(a.prog, xv, yv, yt);
             for (int k = 0; k < a.m; ++k) {
                 S::store1(static_cast<E*>(a.y[k]) + i, yv[k][0]);
                 S::store1(static_cast<E*>(a.d[k]) + i, yt[k][0]);
@@ -139,7 +155,8 @@ struct SeqBackwardArgs {
     void* gin;
     int m;
     size_t n;
-    size_t packets;    // whole 16-byte packets handled by the vector loop (0 unless every pointer is 16-byte aligned)
+    size_t head;       // elements before the first 16-byte boundary (the same for every tensor; n if they do not agree)
+    size_t packets;    // whole 16-byte packets after the head
 };
 
 // M is a template parameter so that all 2 M loads of a packet are issued before the first use; a CTA takes one
@@ -152,6 +169,7 @@ __global__ void __launch_bounds__(kBlock, 4) seq_backward_kernel(const SeqBackwa
     using E = typename S::elem;
     constexpr int V = S::kVec;
     constexpr int U = seq_bwd_unroll(M);
+    const size_t byte_off = a.head * sizeof(E);
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     asm volatile("griddepcontrol.wait;" ::: "memory");
     const size_t tile = size_t(kBlock) * U;
@@ -163,8 +181,8 @@ __global__ void __launch_bounds__(kBlock, 4) seq_backward_kernel(const SeqBackwa
             if (pk < a.packets) {
 #pragma unroll
                 for (int k = 0; k < M; ++k) {
-                    rg[u][k] = load_packet(static_cast<const uint4*>(a.g[k]) + pk);
-                    rd[u][k] = load_packet(static_cast<const uint4*>(a.d[k]) + pk);
+                    rg[u][k] = load_packet(reinterpret_cast<const uint4*>(static_cast<const char*>(a.g[k]) + byte_off) + pk);
+                    rd[u][k] = load_packet(reinterpret_cast<const uint4*>(static_cast<const char*>(a.d[k]) + byte_off) + pk);
                 }
             }
         }
@@ -184,11 +202,14 @@ __global__ void __launch_bounds__(kBlock, 4) seq_backward_kernel(const SeqBackwa
 #pragma unroll
                 for (int e = 0; e < V; ++e) acc[e] = fmaf(gv[e], dv[e], acc[e]);
             }
-            *(static_cast<uint4*>(a.gin) + pk) = S::pack(acc);
+            *(reinterpret_cast<uint4*>(static_cast<char*>(a.gin) + byte_off) + pk) = S::pack(acc);
         }
     }
-    if (blockIdx.x == 0) {
-        for (size_t i = a.packets * V + threadIdx.x; i < a.n; i += kBlock) {
+    {   // outside the packet grid: spread over the whole grid (see seq_forward_kernel)
+        const size_t tail_begin = a.head + a.packets * V;
+        const size_t n_edge = a.head + (a.n - tail_begin);
+        for (size_t j = size_t(blockIdx.x) * kBlock + threadIdx.x; j < n_edge; j += size_t(gridDim.x) * kBlock) {
+            const size_t i = j < a.head ? j : tail_begin + (j - a.head);
             float acc = S::load1(static_cast<const E*>(a.g[0]) + i) * S::load1(static_cast<const E*>(a.d[0]) + i);
 #pragma unroll
             for (int k = 1; k < M; ++k)
@@ -211,12 +232,14 @@ struct EwArgs {
     int backward;
     float c;
     size_t n;
-    size_t packets;    // as in SeqBackwardArgs
+    size_t head, packets;    // as in SeqBackwardArgs
 };
 
+template <class P>
 __device__ __forceinline__ void ew_apply(int op, int backward, float c, float i0, float i1, float i2, float& o0, float& o1)
 {
-    const Dual<Fast> a{i0, 0.0f};
+    using T = typename ScalarOf<P>::type;
+    const Dual<P> a{T(i0), T(0)};
     o1 = 0.0f;
     if (!backward) {
         switch (op) {
@@ -224,30 +247,33 @@ __device__ __forceinline__ void ew_apply(int op, int backward, float c, float i0
         case kSeqMul: o0 = i0 * i1; break;
         case kSeqScale: o0 = c * i0; break;
         case kSeqAddConst: o0 = c + i0; break;
-        case kSeqExp: o0 = dual_exp(a).v; break;
-        case kSeqLog1p: o0 = dual_log1p(a).v; break;
-        case kSeqTanh: o0 = dual_tanh(a).v; break;
-        case kSeqErf: o0 = dual_erf(a).v; break;
-        case kSeqSoftplus: o0 = dual_softplus(a).v; break;
-        case kSeqSigmoid: o0 = dual_sigmoid(a).v; break;
-        case kSeqHalfOnePlusTanh: o0 = dual_half_one_plus_tanh(a).v; break;
-        case kSeqHalfOnePlusErf: o0 = dual_half_one_plus_erf(a).v; break;
+        case kSeqExp: o0 = dual_value(dual_exp(a)); break;
+        case kSeqLog1p: o0 = dual_value(dual_log1p(a)); break;
+        case kSeqTanh: o0 = dual_value(dual_tanh(a)); break;
+        case kSeqErf: o0 = dual_value(dual_erf(a)); break;
+        case kSeqSoftplus: o0 = dual_value(dual_softplus(a)); break;
+        case kSeqSigmoid: o0 = dual_value(dual_sigmoid(a)); break;
+        case kSeqHalfOnePlusTanh: o0 = dual_value(dual_half_one_plus_tanh(a)); break;
+        case kSeqHalfOnePlusErf: o0 = dual_value(dual_half_one_plus_erf(a)); break;
         default: o0 = i0; break;
         }
     } else {
-        // i0 = upstream gradient; i1, i2 = what the rule kept
+        // i0 = upstream gradient; i1, i2 = what the rule kept.  The rule's own factor is the tangent that the
+        // primitive returns for a unit input tangent, wherever the rule keeps the operator's INPUT; where it keeps the
+        // OUTPUT the factor is the usual closed form in that output.
         const float g = i0;
+        const Dual<P> in{T(i1), T(1)};
         switch (op) {
         case kSeqMul: o0 = g * i2; o1 = g * i1; break;                        // kept: both operands
         case kSeqScale: o0 = c * g; break;
         case kSeqExp: o0 = g * i1; break;                                     // kept: the output
-        case kSeqLog1p: o0 = g * hw::rcp_approx(1.0f + i1); break;            // kept: the input
+        case kSeqLog1p: o0 = g * dual_tangent(dual_log1p(in)); break;         // kept: the input
         case kSeqTanh: o0 = g * fmaf(-i1, i1, 1.0f); break;                   // kept: the output
-        case kSeqErf: o0 = g * (1.12837923f * hw::ex2_approx(-1.44269502f * (i1 * i1))); break;      // input
-        case kSeqSoftplus: o0 = g * dual_sigmoid(Dual<Fast>{i1, 0.0f}).v; break;                     // input
+        case kSeqErf: o0 = g * dual_tangent(dual_erf(in)); break;             // input
+        case kSeqSoftplus: o0 = g * dual_tangent(dual_softplus(in)); break;   // input
         case kSeqSigmoid: o0 = g * (i1 * (1.0f - i1)); break;                 // kept: the output
         case kSeqHalfOnePlusTanh: o0 = g * ((i1 + i1) * (1.0f - i1)); break;  // kept: the output
-        case kSeqHalfOnePlusErf: o0 = g * (0.564189613f * hw::ex2_approx(-1.44269502f * (i1 * i1))); break;   // input
+        case kSeqHalfOnePlusErf: o0 = g * dual_tangent(dual_half_one_plus_erf(in)); break;   // input
         default: o0 = g; break;
         }
     }
@@ -264,6 +290,7 @@ __global__ void __launch_bounds__(kBlock, 4) ew_kernel(const EwArgs a)
     using E = typename S::elem;
     constexpr int V = S::kVec;
     constexpr int U = kEwUnroll;
+    const size_t byte_off = a.head * sizeof(E);
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     asm volatile("griddepcontrol.wait;" ::: "memory");
     const size_t tile = size_t(kBlock) * U;
@@ -273,9 +300,9 @@ __global__ void __launch_bounds__(kBlock, 4) ew_kernel(const EwArgs a)
         for (int u = 0; u < U; ++u) {
             const size_t pk = base + size_t(u) * kBlock;
             if (pk < a.packets) {
-                r0[u] = load_packet(static_cast<const uint4*>(a.in[0]) + pk);
-                if (a.in[1]) r1[u] = load_packet(static_cast<const uint4*>(a.in[1]) + pk);
-                if (a.in[2]) r2[u] = load_packet(static_cast<const uint4*>(a.in[2]) + pk);
+                r0[u] = load_packet(reinterpret_cast<const uint4*>(static_cast<const char*>(a.in[0]) + byte_off) + pk);
+                if (a.in[1]) r1[u] = load_packet(reinterpret_cast<const uint4*>(static_cast<const char*>(a.in[1]) + byte_off) + pk);
+                if (a.in[2]) r2[u] = load_packet(reinterpret_cast<const uint4*>(static_cast<const char*>(a.in[2]) + byte_off) + pk);
             }
         }
 #pragma unroll
@@ -287,18 +314,21 @@ __global__ void __launch_bounds__(kBlock, 4) ew_kernel(const EwArgs a)
             if (a.in[1]) S::unpack(r1[u], i1);
             if (a.in[2]) S::unpack(r2[u], i2);
 #pragma unroll
-            for (int e = 0; e < V; ++e) ew_apply(OP, BWD, a.c, i0[e], a.in[1] ? i1[e] : 0.0f, a.in[2] ? i2[e] : 0.0f, o0[e], o1[e]);
-            *(static_cast<uint4*>(a.out[0]) + pk) = S::pack(o0);
-            if (a.out[1]) *(static_cast<uint4*>(a.out[1]) + pk) = S::pack(o1);
+            for (int e = 0; e < V; ++e) ew_apply<typename SeqPolicy<S>::type>(OP, BWD, a.c, i0[e], a.in[1] ? i1[e] : 0.0f, a.in[2] ? i2[e] : 0.0f, o0[e], o1[e]);
+            *(reinterpret_cast<uint4*>(static_cast<char*>(a.out[0]) + byte_off) + pk) = S::pack(o0);
+            if (a.out[1]) *(reinterpret_cast<uint4*>(static_cast<char*>(a.out[1]) + byte_off) + pk) = S::pack(o1);
         }
     }
-    if (blockIdx.x == 0) {
-        for (size_t i = a.packets * V + threadIdx.x; i < a.n; i += kBlock) {
+    {   // outside the packet grid: spread over the whole grid (see seq_forward_kernel)
+        const size_t tail_begin = a.head + a.packets * V;
+        const size_t n_edge = a.head + (a.n - tail_begin);
+        for (size_t j = size_t(blockIdx.x) * kBlock + threadIdx.x; j < n_edge; j += size_t(gridDim.x) * kBlock) {
+            const size_t i = j < a.head ? j : tail_begin + (j - a.head);
             float i0 = S::load1(static_cast<const E*>(a.in[0]) + i);
             float i1 = a.in[1] ? S::load1(static_cast<const E*>(a.in[1]) + i) : 0.0f;
             float i2 = a.in[2] ? S::load1(static_cast<const E*>(a.in[2]) + i) : 0.0f;
             float o0, o1;
-            ew_apply(OP, BWD, a.c, i0, i1, i2, o0, o1);
+            ew_apply<typename SeqPolicy<S>::type>(OP, BWD, a.c, i0, i1, i2, o0, o1);
             S::store1(static_cast<E*>(a.out[0]) + i, o0);
             if (a.out[1]) S::store1(static_cast<E*>(a.out[1]) + i, o1);
         }

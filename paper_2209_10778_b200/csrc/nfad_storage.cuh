@@ -27,7 +27,7 @@ namespace nfad {
 #define NFAD_MIN_BLOCKS_16 5
 #endif
 #ifndef NFAD_MIN_BLOCKS_32
-#define NFAD_MIN_BLOCKS_32 5
+#define NFAD_MIN_BLOCKS_32 4
 #endif
 
 // ---------------------------------------------------------------- storage types

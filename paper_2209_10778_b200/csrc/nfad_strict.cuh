@@ -15,7 +15,7 @@
 
 namespace nfad {
 
-// The argument is already clamped to [-kFull, 0): all exponentials stay finite and non-zero where it matters.
+// The argument is already clamped to [-kWide, 0): all exponentials stay finite and non-zero where it matters.
 __device__ __forceinline__ double fprime_negative_f64(GeluErf, double x)
 {
     const double kInvSqrt2 = 0.70710678118654752440, kInvSqrt2Pi = 0.39894228040143267794;
@@ -56,12 +56,12 @@ __device__ __forceinline__ double fprime_negative_f64(Mish, double x)
 }
 
 // x -> (f(x), f'(x)): the value and, for x >= 0, the derivative from the regular fp32-storage chain
-// (already within 4 ulp of themselves there); the derivative for x < 0 from fp64.
+// (within a rounding of themselves there); the derivative for x < 0 from the forms above.
 template <class K> __device__ __forceinline__ ActOut evaluate_strict(float x)
 {
-    ActOut o = evaluate(K{}, Full{}, x);
+    ActOut o = evaluate(K{}, Wide{}, x);
     if (x < 0.0f) {
-        constexpr float kSat = Saturation<K>::kFull;
+        constexpr float kSat = Saturation<K>::kWide;
         o.dydx = __double2float_rn(fprime_negative_f64(K{}, (double)fmaxf(x, -kSat)));
     }
     return o;

@@ -255,7 +255,7 @@ def test_tall_narrow_tensor_covers_the_row_chunk_loop():
 
 
 @pytest.mark.parametrize("dtype", DTYPES)
-def test_value_only_forward_gives_the_training_value(dtype):
+def test_value_only_forward_against_the_training_value(dtype):
     for rows, cols in ((300, 768), (41, 1003)):
         x = W.normal(rows * cols, dtype, 81, 1.5, DEV)
         bias = W.normal(cols, dtype, 82, 0.5, DEV)
@@ -264,7 +264,10 @@ def test_value_only_forward_gives_the_training_value(dtype):
             nfad.nfad_bias_act_forward(kind, x, bias, y, d)
             nfad.nfad_bias_act_forward_infer(kind, x, bias, yi)
             torch.cuda.synchronize()
-            assert np.array_equal(W.raw_numpy(y), W.raw_numpy(yi)), (kind, dtype, rows, cols)
+            if kind == "gelu_erf" and dtype != "f32":     # the 16-bit erf gate has a cheaper value-only form: one ulp at most
+                assert (ulp.ulp_distance16(W.raw_numpy(y), W.raw_numpy(yi)) <= 1).all(), (kind, dtype, rows, cols)
+            else:
+                assert np.array_equal(W.raw_numpy(y), W.raw_numpy(yi)), (kind, dtype, rows, cols)
     xs = torch.tensor([float("inf"), float("-inf"), float("nan"), 0.0], device=DEV, dtype=W.TORCH_DTYPES[dtype])
     b1 = torch.zeros(4, device=DEV, dtype=W.TORCH_DTYPES[dtype])
     out = torch.empty_like(xs)

@@ -104,14 +104,27 @@ def test_backward_extreme_values(dtype):
 
 @pytest.mark.parametrize("kind", KINDS)
 @pytest.mark.parametrize("dtype", ["f32", "bf16", "f16"])
-def test_infer_equals_training_value(kind, dtype):
+def test_infer_against_the_oracle_and_the_training_value(kind, dtype):
+    """The value-only pass is held to the oracle like the training pass.  It gives the training pass's very bits wherever it
+    runs the same chain; the 16-bit erf gate has a cheaper value-only form (a lower-degree fit, good to a quarter of an fp16
+    ulp), whose results may differ from the training value by one unit in the last place, never more."""
     n = 70001
     x = W.draw("mix", n, dtype, 7, DEV)
     y, _ = parity.gpu_forward(kind, x)
     y2 = torch.empty_like(x)
     nfad.nfad_act_forward_infer(kind, x, y2)
     torch.cuda.synchronize()
-    assert np.array_equal(W.raw_numpy(y), W.raw_numpy(y2))
+    x_raw, y2_raw = W.raw_numpy(x), W.raw_numpy(y2)
+    if dtype == "f32":
+        assert np.array_equal(W.raw_numpy(y), y2_raw)
+    else:
+        f, _ = oracle.forward(kind, dtype, x_raw)
+        dist = ulp.ulp_distance16(y2_raw, oracle.round_to(dtype, f))
+        assert (dist <= 1).all() and not ulp.is_nan16(y2_raw, dtype).any()
+        if kind == "gelu_erf":
+            assert (ulp.ulp_distance16(y2_raw, W.raw_numpy(y)) <= 1).all()
+        else:
+            assert np.array_equal(W.raw_numpy(y), y2_raw)
 
 
 @pytest.mark.parametrize("kind", KINDS)

@@ -200,7 +200,10 @@ def test_autograd_wrappers():
         y2 = nfad_autograd.ConventionalActivation.apply(x2, kind)
         y2.backward(g)
         torch.cuda.synchronize()
-        assert torch.equal(y2.detach(), y.detach())
+        if kind == "gelu_erf":      # the 16-bit erf gate has a cheaper value-only form: one unit in the last place at most
+            assert (ulp.ulp_distance16(W.raw_numpy(y2.detach()), W.raw_numpy(y.detach())) <= 1).all()
+        else:
+            assert torch.equal(y2.detach(), y.detach())
         assert torch.allclose(x2.grad.float(), x.grad.float(), rtol=2e-2, atol=1e-3)
     # a two-result sequence through autograd
     prog = _two_result_program()
@@ -258,3 +261,60 @@ def test_four_results_forward_and_backward(dtype, executor):
     got = oracle.widen(dtype, W.raw_numpy(gin))
     tol = (2.0 ** -22 if dtype == "f32" else 2.0 ** -7) * want_abs + 1e-30
     assert (np.abs(got - want) <= tol).all()
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_large_sliced_views_use_the_whole_device(dtype, executor):
+    """A view that starts one element into an allocation (every tensor sliced alike: one common offset modulo 16 bytes) and
+    views that share no offset (no packet grid at all) give the same bits as aligned tensors, and the second case -- where
+    every element goes through the element-wise path -- must not crawl through one CTA: it is timed against the aligned run."""
+    prog = _two_result_program()
+    td = W.TORCH_DTYPES[dtype]
+    n = (1 << 22) + 3
+    base = W.normal(n + 8, dtype, 31, 1.5, DEV)
+    gbase = [W.normal(n + 8, dtype, 32 + k, 1.0, DEV) for k in range(2)]
+
+    def run(ox, oy, od, og):
+        x = base[ox:ox + n]
+        ys = [torch.empty(n + 8, dtype=td, device=DEV)[oy:oy + n] for _ in range(2)]
+        ds = [torch.empty(n + 8, dtype=td, device=DEV)[od:od + n] for _ in range(2)]
+        gs = [g[og:og + n] for g in gbase]
+        gin = torch.empty(n + 8, dtype=td, device=DEV)[ox:ox + n]
+        nfad.nfad_seq_forward(prog.ops, x, ys, ds)                # warm-up (and compilation)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        nfad.nfad_seq_forward(prog.ops, x, ys, ds)
+        nfad.nfad_seq_backward(gs, ds, gin)
+        e1.record()
+        torch.cuda.synchronize()
+        # a third tensor through the one-operator kernels on the same views
+        t = torch.empty(n + 8, dtype=td, device=DEV)[oy:oy + n]
+        nfad.nfad_ew_op("tanh", False, 0.0, x, None, None, t)
+        torch.cuda.synchronize()
+        return [W.raw_numpy(v) for v in ys + ds + [t]], W.raw_numpy(gin), e0.elapsed_time(e1)
+
+    ref, gin_ref, ms_ref = run(0, 0, 0, 0)
+    same, gin_same, _ = run(1, 1, 1, 1)
+    # x shifted by one element: compare against a reference computed from that very view
+    x1 = base[1:1 + n].clone()                                   # aligned copy of the shifted view
+    ys1 = [torch.empty(n, dtype=td, device=DEV) for _ in range(2)]
+    ds1 = [torch.empty(n, dtype=td, device=DEV) for _ in range(2)]
+    nfad.nfad_seq_forward(prog.ops, x1, ys1, ds1)
+    t1 = torch.empty(n, dtype=td, device=DEV)
+    nfad.nfad_ew_op("tanh", False, 0.0, x1, None, None, t1)
+    torch.cuda.synchronize()
+    want1 = [W.raw_numpy(v) for v in ys1 + ds1 + [t1]]
+    for a, b in zip(same, want1):
+        assert np.array_equal(a, b)
+    gin1 = torch.empty(n, dtype=td, device=DEV)
+    nfad.nfad_seq_backward([g[1:1 + n].clone() for g in gbase], ds1, gin1)
+    torch.cuda.synchronize()
+    assert np.array_equal(gin_same, W.raw_numpy(gin1))
+    mixed, gin_mixed, ms_mixed = run(1, 2, 3, 1)                  # three different offsets: no common packet grid
+    for a, b in zip(mixed, want1):
+        assert np.array_equal(a, b)
+    assert np.array_equal(gin_mixed, W.raw_numpy(gin1))
+    assert nfad.nfad_seq_last_executor() == executor
+    # the element-wise path over the whole grid costs a small multiple of the packet path, not the ~10^3 of one CTA
+    assert ms_mixed < 40 * ms_ref, (ms_mixed, ms_ref)
