@@ -354,8 +354,11 @@ NFAD_API size_t nfad_bias_act_backward_scratch_bytes(int dtype, size_t rows, siz
  * order too (the copies start when `stream` reaches the call).  flags = NFAD_HOST_INPUTS_READY: the
  * caller guarantees that x_host and grad_out_host hold their final contents when the call is made
  * and that no work pending on `stream` writes them; the input copies may then start at once, so
- * that consecutive calls keep both directions of the link busy across the call boundary (a call
- * whose workspace or chunk size differs from the previous one's first waits for that one to finish).
+ * that consecutive calls keep both directions of the link busy across the call boundary.  Calls on
+ * one device share the pipeline, whatever stream they name: the copies of a later call run after
+ * those of an earlier one, and with either flag value a call whose workspace or chunk size differs
+ * from the previous call's first waits until that call has finished with its workspace, so two
+ * callers on different streams may not corrupt each other's slots (they do take turns).
  * Any other flag bit gives NFAD_E_LAYOUT.  State: two streams and a few events per
  * device, created on the first call on that device (make that call outside a stream capture; the
  * call itself cannot be captured into a graph) and kept until the process exits; enqueueing is

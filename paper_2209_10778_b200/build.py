@@ -62,10 +62,9 @@ def build_library(force: bool = False, verbose: bool = False) -> str:
     nvcc = _nvcc()
     objs = []
     procs = []
-    tuning = os.environ.get("NFAD_NVCC_FLAGS", "").split()     # e.g. -DNFAD_UNROLL=2, for experiments
     for src, extra in UNITS:
         obj = os.path.join(OBJ_DIR, src.replace(".cu", ".o"))
-        cmd = [nvcc, *ARCH, *COMMON, *extra, *tuning, "-c", os.path.join(CSRC, src), "-o", obj]
+        cmd = [nvcc, *ARCH, *COMMON, *extra, "-c", os.path.join(CSRC, src), "-o", obj]
         if verbose:
             cmd.insert(1, "-Xptxas=-v")
             print(" ".join(cmd), flush=True)

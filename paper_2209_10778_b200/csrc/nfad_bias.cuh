@@ -34,12 +34,8 @@ constexpr int kBiasMaxBlock = 256;
 
 // Threads per CTA: the multiple of 32 in [64, 256] that leaves the fewest idle lanes in the last strip
 // of a row (the largest such on a tie).
-#ifndef NFAD_BIAS_BLOCK
-#define NFAD_BIAS_BLOCK 0
-#endif
 inline unsigned bias_block(size_t row_packets)
 {
-    if (NFAD_BIAS_BLOCK) return NFAD_BIAS_BLOCK;
     unsigned best = kBiasMaxBlock;
     size_t best_waste = ~size_t(0);
     for (unsigned b = kBiasMaxBlock; b >= 64; b -= 32) {
@@ -61,7 +57,7 @@ inline void bias_launch_config(cudaLaunchConfig_t* cfg, cudaLaunchAttribute* att
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg->attrs = attr;
-    cfg->numAttrs = (pdl && NFAD_PDL) ? 1 : 0;
+    cfg->numAttrs = pdl ? 1 : 0;
 }
 
 // ---------------------------------------------------------------- forward
@@ -109,10 +105,8 @@ __global__ void __launch_bounds__(kBiasMaxBlock, S::kMinBlocks) bias_forward_ker
 {
     constexpr int V = S::kVec;
     constexpr int U = kBiasRows;
-#if NFAD_PDL
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     asm volatile("griddepcontrol.wait;" ::: "memory");
-#endif
     const uint4* x4 = static_cast<const uint4*>(a.x);
     uint4* y4 = static_cast<uint4*>(a.y);
     uint4* d4 = static_cast<uint4*>(a.d);
@@ -211,17 +205,12 @@ struct BiasBackwardArgs {
     uint32_t chunk_rows;     // rows per chunk
 };
 
-// How the rows are cut into chunks: enough CTAs to fill the device NFAD_BIAS_WAVES times over,
+// How the rows are cut into chunks: enough CTAs to fill the device kBiasWaves times over,
 // never fewer than kBiasRows rows per chunk, at most kBiasMaxChunks chunks.  The plan depends on
 // the shape, the storage type and the device only -- not on pointer alignment -- so that the
 // vector and the element-wise kernels add the same numbers in the same order.
-#ifndef NFAD_BIAS_MAX_CHUNKS
-#define NFAD_BIAS_MAX_CHUNKS 256
-#endif
-#ifndef NFAD_BIAS_WAVES
-#define NFAD_BIAS_WAVES 2
-#endif
-constexpr int kBiasMaxChunks = NFAD_BIAS_MAX_CHUNKS;
+constexpr int kBiasMaxChunks = 256;
+constexpr int kBiasWaves = 2;
 
 struct BiasPlan { unsigned block; uint32_t strips, chunks, chunk_rows; };
 
@@ -233,7 +222,7 @@ inline BiasPlan bias_plan(size_t rows, size_t cols, int sm_count)
     p.block = bias_block(row_packets);
     p.strips = uint32_t((row_packets + p.block - 1) / p.block);
     if (p.strips == 0) p.strips = 1;
-    const size_t target = size_t(sm_count) * (1024 / p.block) * NFAD_BIAS_WAVES;
+    const size_t target = size_t(sm_count) * (1024 / p.block) * kBiasWaves;
     size_t chunks = (target + p.strips - 1) / p.strips;
     const size_t max_by_rows = (rows + kBiasRows - 1) / kBiasRows;
     if (chunks > max_by_rows) chunks = max_by_rows;
@@ -253,10 +242,8 @@ __global__ void __launch_bounds__(kBiasMaxBlock, 4) bias_backward_kernel(const B
 {
     constexpr int V = S::kVec;
     constexpr int U = kBiasRows;
-#if NFAD_PDL
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     asm volatile("griddepcontrol.wait;" ::: "memory");
-#endif
     const uint4* g4 = static_cast<const uint4*>(a.g);
     const uint4* d4 = static_cast<const uint4*>(a.d);
     uint4* o4 = static_cast<uint4*>(a.gin);
@@ -332,9 +319,7 @@ static __global__ void __launch_bounds__(32 * kBiasGroups) bias_reduce_chunks_ke
                                                                                      uint32_t chunks, uint32_t cols)
 {
     __shared__ float smem[kBiasGroups][32];
-#if NFAD_PDL
     asm volatile("griddepcontrol.wait;" ::: "memory");
-#endif
     const int lane = threadIdx.x & 31, group = threadIdx.x >> 5;
     const size_t col = size_t(blockIdx.x) * 32 + lane;
     const uint32_t per = (chunks + kBiasGroups - 1) / kBiasGroups;

@@ -280,7 +280,7 @@ NFAD_DEV Gate<Fast> gate(Fast, GeluTanh, Seed X)
 }
 NFAD_DEV Gate<Wide> gate(Wide, GeluTanh, Seed X)
 {
-    return dual_half_one_plus_tanh(dual_odd_cubic(Wide{}, 0.7978845608028654, 0.035677408136300125, 0.10703222440890037, X));
+    return dual_half_one_plus_tanh(InRange{}, dual_odd_cubic(Wide{}, 0.7978845608028654, 0.035677408136300125, 0.10703222440890037, X));
 }
 
 // Swish (Table I, Table II): h = sigmoid(x)

@@ -36,7 +36,7 @@ template <int kSteps = 2> NFAD_DEV double rcp(double d)
 // e^a for |a| <= 700: a = n ln2 + r with |r| <= ln2/2 (n taken from the low word of a sum with 1.5 * 2^52), a minimax
 // polynomial for e^r, and 2^n added into the exponent field (the result stays normal for |a| <= 700; every caller keeps
 // its argument inside that).  Degree 6 leaves a relative error of 2^-29 (a thirtieth of an fp32 ulp: what the four
-// activations need), degree 8 of 2^-39.8 (the general-purpose primitives).
+// activations need), degree 11 of 2^-55 (the general-purpose primitives, whose results other operations may cancel).
 template <int kDegree> NFAD_DEV double exp_bounded(double a)
 {
     const double kMagic = 6755399441055744.0;
@@ -44,6 +44,7 @@ template <int kDegree> NFAD_DEV double exp_bounded(double a)
     double n = t - kMagic;
     int ni = hw::double_lo(t);
     double r = fma(n, -0.6931471805599453, a);
+    if (kDegree != 6) r = fma(n, -2.3190468138462996e-17, r);      // the rest of ln2: |n| reaches 1000
     double p;
     if (kDegree == 6) {
         p = 0.0013836846134577057;
@@ -54,43 +55,44 @@ template <int kDegree> NFAD_DEV double exp_bounded(double a)
         p = fma(p, r, 1.0000000363231765);
         p = fma(p, r, 1.0000000005541663);
     } else {
-        p = 2.487623871994097e-05;
-        p = fma(p, r, 0.00019915941664891244);
-        p = fma(p, r, 0.0013888821542986098);
-        p = fma(p, r, 0.008333265963232838);
-        p = fma(p, r, 0.041666666891631156);
-        p = fma(p, r, 0.16666666891720291);
-        p = fma(p, r, 0.49999999999797123);
-        p = fma(p, r, 0.9999999999797041);
+        p = 2.5110095611886237e-08;
+        p = fma(p, r, 2.7632715071632255e-07);
+        p = fma(p, r, 2.7557240761739257e-06);
+        p = fma(p, r, 2.4801485278370062e-05);
+        p = fma(p, r, 0.00019841269890193705);
+        p = fma(p, r, 0.0013888888952505406);
+        p = fma(p, r, 0.008333333333319546);
+        p = fma(p, r, 0.04166666666648738);
+        p = fma(p, r, 0.1666666666666668);
+        p = fma(p, r, 0.5000000000000019);
+        p = fma(p, r, 1.0);
         p = fma(p, r, 1.0);
     }
     return hw::double_from(hw::double_hi(p) + (ni << 20), hw::double_lo(p));
 }
-NFAD_DEV double exp_neg(double a) { return exp_bounded<8>(a); }
+NFAD_DEV double exp_neg(double a) { return exp_bounded<11>(a); }
 
 // erfc(z)/2 = exp(-z^2) W(z) for z >= 0.  W(z) (z + k) is a smooth function of q = (z - k)/(z + k) in [-1, 1), fitted
-// by one degree-10 polynomial on z in [0, 15], k = 3/sqrt(2).  Returns W(z); the caller owns the exponential, so that
-// value and slope share it.
-//   half_erfcx:     everything in double (relative error 2^-27.7, the fit's), for the general-purpose erf;
+// by one polynomial on z in [0, 15], k = 3/sqrt(2).  Returns W(z); the caller owns the exponential, so that value and
+// slope share it.
+//   half_erfcx:     everything in double, degree 22 (relative error 2^-52, the arithmetic's), for the general-purpose erf;
 //   half_erfcx_mix: r = 1/(z + k) and the final product in double, the polynomial itself in fp32 on the otherwise idle
 //                   fp32 pipe (q in (-1, 1) and a result in [0.28, 1.07] make that a well-conditioned Horner chain: the
 //                   result is good to about 0.8 fp32 ulp, which the activations' tolerance has room for).
 NFAD_DEV double half_erfcx(double z)
 {
     const double k = 2.1213202476501465;
-    double r = rcp<1>(z + k);
+    const double c[23] = {0.5155400178331069, -0.3601520858466969, 0.16264707189352245, -0.03341999312315092, -0.007398367634744453,
+                          0.004930386718851745, 0.0007266182227491928, -0.0007395124001504905, -0.0001814263229256693,
+                          0.00010917379216550876, 5.572919709637488e-05, -9.368798767498136e-06, -1.4631205627619127e-05,
+                          -2.479590212362355e-06, 2.582014193120429e-06, 1.580743084650836e-06, -1.5835451846490903e-08,
+                          -4.0458837978587706e-07, -1.5996308446846036e-07, 2.7211538400833845e-08, 3.937772165516381e-08,
+                          1.0068658595420031e-08, 4.3545861799549443e-10};
+    double r = rcp<2>(z + k);
     double q = fma(-2.0 * k, r, 1.0);
-    double p = 3.897072125339127e-05;
-    p = fma(p, q, 9.319733096317181e-05);
-    p = fma(p, q, -0.0001739974147955117);
-    p = fma(p, q, -0.0007308700486527253);
-    p = fma(p, q, 0.0007252048472983968);
-    p = fma(p, q, 0.0049284903718876845);
-    p = fma(p, q, -0.007398255674427253);
-    p = fma(p, q, -0.0334198465781627);
-    p = fma(p, q, 0.16264706813819155);
-    p = fma(p, q, -0.3601520876697053);
-    p = fma(p, q, 0.5155400178703385);
+    double p = c[22];
+#pragma unroll
+    for (int i = 21; i >= 0; --i) p = fma(p, q, c[i]);
     return p * r;
 }
 NFAD_DEV double half_erfcx_mix(double z_plus_k)
@@ -120,7 +122,7 @@ NFAD_DEV double log_pos(double u)
     int mh = (hi & 0x000fffff) | 0x3ff00000;
     if (mh >= 0x3ff6a09e) { mh -= 0x00100000; k += 1; }     // m >= sqrt(2): halve it
     double m = hw::double_from(mh, hw::double_lo(u));
-    double s = (m - 1.0) * rcp(m + 1.0);
+    double s = (m - 1.0) * rcp<2>(m + 1.0);
     double s2 = s * s;
     double p = 0.13333333333333333;                           // 2/15
     p = fma(p, s2, 0.15384615384615385);
@@ -150,50 +152,50 @@ NFAD_DEV Dual<Wide> as_dual(const Gate<Wide>& a) { return {a.v, a.t}; }
 NFAD_DEV Dual<Wide> dual_add(const Dual<Wide>& a, const Dual<Wide>& b) { return {a.v + b.v, a.t + b.t}; }
 NFAD_DEV Dual<Wide> dual_add_const(double c, const Dual<Wide>& a) { return {c + a.v, a.t}; }
 NFAD_DEV Dual<Wide> dual_scale(double c, const Dual<Wide>& a) { return {c * a.v, c * a.t}; }
-NFAD_DEV Dual<Wide> dual_scale(Wide, double c, const Seed& a) { return {c * double(a.x), c}; }
-NFAD_DEV Dual<Wide> dual_mul(Wide, const Seed& a, const Seed& b) { return {double(a.x) * double(b.x), double(a.x) + double(b.x)}; }
-NFAD_DEV Dual<Wide> dual_mul(const Seed& a, const Dual<Wide>& b) { return {double(a.x) * b.v, fma(double(a.x), b.t, b.v)}; }
-NFAD_DEV Gate<Wide> dual_mul(const Seed& a, const Gate<Wide>& b) { return {double(a.x) * b.v, fma(double(a.x), b.t, b.v)}; }
+NFAD_DEV Dual<Wide> dual_scale(Wide, double c, const Seed& a) { return {c * hw::to_double(a.x), c}; }
+NFAD_DEV Dual<Wide> dual_mul(Wide, const Seed& a, const Seed& b) { return {hw::to_double(a.x) * hw::to_double(b.x), hw::to_double(a.x) + hw::to_double(b.x)}; }
+NFAD_DEV Dual<Wide> dual_mul(const Seed& a, const Dual<Wide>& b) { return {hw::to_double(a.x) * b.v, fma(hw::to_double(a.x), b.t, b.v)}; }
+NFAD_DEV Gate<Wide> dual_mul(const Seed& a, const Gate<Wide>& b) { return {hw::to_double(a.x) * b.v, fma(hw::to_double(a.x), b.t, b.v)}; }
 NFAD_DEV Dual<Wide> dual_mul(const Dual<Wide>& a, const Dual<Wide>& b) { return {a.v * b.v, fma(a.v, b.t, a.t * b.v)}; }
 
 // c1 x + c3 x^3 with tangent c1 + k3 x^2 (k3 = 3 c3)
 NFAD_DEV Dual<Wide> dual_odd_cubic(Wide, double c1, double c3, double k3, const Seed& a)
 {
-    double x = double(a.x);
+    double x = hw::to_double(a.x);
     double s = x * x;
     return {x * fma(c3, s, c1), fma(k3, s, c1)};
 }
 
-NFAD_DEV Dual<Wide> as_wide(const Seed& a) { return {double(a.x), 1.0}; }
+NFAD_DEV Dual<Wide> as_wide(const Seed& a) { return {hw::to_double(a.x), 1.0}; }
 NFAD_DEV Dual<Wide> as_wide(const Dual<Wide>& a) { return a; }
 
 // ----------------------------------------------------------------- the logistic gates
 
 // L(w) = 1/(1 + exp(-w)) and dL/dw = L (1 - L), one form for both signs: E = exp(-w), L = 1/(1 + E), 1 - L = E L
 // (no subtraction anywhere; doubles have the range for E on either side).  The slope is returned times `slope_in`
-// (the chain rule's next factor).  |w| <= 700.
-NFAD_DEV Gate<Wide> logistic_wide(double w, double slope_in)
+// (the chain rule's next factor).  |w| <= 700.  kPrecise: the exponential and the reciprocal to 2^-52 instead of 2^-29.
+template <bool kPrecise> NFAD_DEV Gate<Wide> logistic_wide(double w, double slope_in)
 {
-    double E = wide::exp_bounded<6>(-w);
-    double L = wide::rcp<1>(1.0 + E);
+    double E = wide::exp_bounded<kPrecise ? 11 : 6>(-w);
+    double L = wide::rcp<kPrecise ? 2 : 1>(1.0 + E);
     return {L, (L * (E * L)) * slope_in};
 }
+NFAD_DEV double clamp700(double v) { return v != v ? v : fmin(fmax(v, -700.0), 700.0); }
 
-NFAD_DEV Gate<Wide> dual_sigmoid(Wide, const Seed& a) { return logistic_wide(double(a.x), 1.0); }
-NFAD_DEV Gate<Wide> dual_sigmoid(const Dual<Wide>& a)
-{
-    return logistic_wide(a.v != a.v ? a.v : fmin(fmax(a.v, -700.0), 700.0), a.t);
-}
+// of the seed (an activation's own gate: |x| is bounded by its caller) and of any dual (clamped here)
+NFAD_DEV Gate<Wide> dual_sigmoid(Wide, const Seed& a) { return logistic_wide<false>(hw::to_double(a.x), 1.0); }
+NFAD_DEV Gate<Wide> dual_sigmoid(const Dual<Wide>& a) { return logistic_wide<true>(clamp700(a.v), a.t); }
 
 // (1 + tanh u)/2 = L(2u), slope 2 L'(2u)
-NFAD_DEV Gate<Wide> dual_half_one_plus_tanh(const Dual<Wide>& u) { return logistic_wide(u.v + u.v, u.t + u.t); }
+NFAD_DEV Gate<Wide> dual_half_one_plus_tanh(InRange, const Dual<Wide>& u) { return logistic_wide<false>(u.v + u.v, u.t + u.t); }
+NFAD_DEV Gate<Wide> dual_half_one_plus_tanh(const Dual<Wide>& u) { return logistic_wide<true>(clamp700(u.v + u.v), u.t + u.t); }
 
 // (1 + erf z)/2 = erfc(-z)/2: with E = exp(-z^2) and W = erfcx(|z|)/2 it is E W for z < 0 and 1 - E W for z >= 0;
-// slope E / sqrt(pi).  |z| <= 15.
+// slope E / sqrt(pi).  Beyond |z| = 15 the gate is 0 or 1 and its slope 0 in double precision.
 NFAD_DEV Gate<Wide> dual_half_one_plus_erf(const Dual<Wide>& z)
 {
-    double za = fabs(z.v);
-    double E = wide::exp_bounded<8>(-(za * za));
+    double za = z.v != z.v ? z.v : fmin(fabs(z.v), 15.0);
+    double E = wide::exp_bounded<11>(-(za * za));
     double a = E * wide::half_erfcx(za);
     return {z.v < 0.0 ? a : 1.0 - a, (E * 0.5641895835477563) * z.t};
 }
@@ -201,13 +203,9 @@ NFAD_DEV Gate<Wide> dual_half_one_plus_erf(const Dual<Wide>& z)
 // Section III-A), so that -c^2 x^2 and c |x| + k each are one operation.  |c x| <= 15.
 NFAD_DEV Gate<Wide> dual_half_one_plus_erf_scaled(Wide, double c, const Seed& a)
 {
-    double x = double(a.x);
+    double x = hw::to_double(a.x);
     double E = wide::exp_bounded<6>((x * x) * -(c * c));
-#if NFAD_ERF_PURE
-    double v = E * wide::half_erfcx(fabs(x) * c);
-#else
     double v = E * wide::half_erfcx_mix(fma(fabs(x), c, 2.1213202476501465));
-#endif
     return {a.x < 0.0f ? v : 1.0 - v, E * (0.5641895835477563 * c)};
 }
 
@@ -215,7 +213,7 @@ NFAD_DEV Gate<Wide> dual_half_one_plus_erf_scaled(Wide, double c, const Seed& a)
 
 // softplus remembers w = exp(v) itself: its slope sigmoid(v) and tanh(softplus) are algebraic in w
 template <> struct SoftplusDual<Wide> { double w; };
-NFAD_DEV SoftplusDual<Wide> dual_softplus(Wide, const Seed& a) { return {wide::exp_bounded<6>(double(a.x))}; }
+NFAD_DEV SoftplusDual<Wide> dual_softplus(Wide, const Seed& a) { return {wide::exp_bounded<6>(hw::to_double(a.x))}; }
 
 // one form for both signs, every term positive:  T = n/(n + 2),  n = w (w + 2),  w = e^v;
 // T' = (dn/dv) 2/(n + 2)^2 = 4 w (w + 1)/(n + 2)^2.  |v| <= 150 keeps (n + 2)^2 inside the range of a double.
@@ -237,7 +235,7 @@ NFAD_DEV Gate<Wide> dual_tanh(const SoftplusDual<Wide>& p)
 NFAD_DEV Dual<Wide> dual_exp(const Dual<Wide>& a)
 {
     double m = wide::exp_neg(-fmin(fabs(a.v), 700.0));
-    double v = a.v > 0.0 ? wide::rcp(m) : m;
+    double v = a.v > 0.0 ? wide::rcp<2>(m) : m;
     v = a.v != a.v ? a.v : v;
     return {v, v * a.t};
 }
@@ -247,8 +245,8 @@ NFAD_DEV Dual<Wide> dual_log1p(const Dual<Wide>& a)
 {
     double u = 1.0 + a.v;
     double um1 = u - 1.0;
-    double v = um1 == 0.0 ? a.v : wide::log_pos(u) * (a.v * wide::rcp(um1));
-    return {v, a.t * wide::rcp(u)};
+    double v = um1 == 0.0 ? a.v : wide::log_pos(u) * (a.v * wide::rcp<2>(um1));
+    return {v, a.t * wide::rcp<2>(u)};
 }
 
 // tanh:  (1 - e)/(1 + e) with e = exp(-2|a|), an odd series below 2^-4 where that cancels; v' = 4e/(1+e)^2.
@@ -256,7 +254,7 @@ NFAD_DEV Dual<Wide> dual_tanh(const Dual<Wide>& a)
 {
     double aa = fmin(fabs(a.v), 350.0);
     double e = wide::exp_neg(-2.0 * aa);
-    double r = wide::rcp(1.0 + e);
+    double r = wide::rcp<2>(1.0 + e);
     double big = (1.0 - e) * r;
     double a2 = aa * aa;
     double ser = fma(a2, fma(a2, fma(a2, fma(a2, 0.021869488536155203, -0.053968253968253971), 0.13333333333333333), -0.33333333333333331), 1.0);
@@ -292,7 +290,7 @@ NFAD_DEV Dual<Wide> dual_softplus(const Dual<Wide>& a)
 {
     double e = wide::exp_neg(-fmin(fabs(a.v), 700.0));
     Dual<Wide> l = dual_log1p(Dual<Wide>{e, 0.0});
-    double r = wide::rcp(1.0 + e);
+    double r = wide::rcp<2>(1.0 + e);
     double v = fmax(a.v, 0.0) + l.v;
     v = a.v != a.v ? a.v : v;
     return {v, (a.v < 0.0 ? e * r : r) * a.t};

@@ -23,13 +23,10 @@ namespace {
 constexpr int kSlots = 4;                      // chunks in flight: one per pipeline stage and one of slack
 constexpr int kMaxDevices = 64;
 constexpr size_t kChunkAlign = 8 * 256;        // elements: whole tiles of the streaming kernels
-#ifndef NFAD_HOST_CHUNK_BYTES
-#define NFAD_HOST_CHUNK_BYTES (size_t(8) << 20)
-#endif
 // Per tensor and slot.  Measured on a 25 MB-per-tensor batch over PCIe 5 x16 (two calls per step, inputs ready):
 // 1 MB chunks reach 6.7, 2 MB 8.4, 4 MB 10.2, 8 MB 11.2 and 16 MB 9.3 G elements/s -- every copy pays a fixed
 // set-up cost, and too few chunks leave nothing to overlap.
-constexpr size_t kPreferredChunkBytes = NFAD_HOST_CHUNK_BYTES;
+constexpr size_t kPreferredChunkBytes = size_t(8) << 20;
 
 struct DeviceState {
     bool ready = false;
@@ -125,8 +122,11 @@ int nfad_host_step(int kind, int dtype, const void* x_host, const void* grad_out
         // fully stream-ordered: the input copies start after whatever the caller's stream holds at this point
         if ((e = cudaEventRecord(s->start, compute)) != cudaSuccess) return fail(e);
         if ((e = cudaStreamWaitEvent(s->h2d, s->start, 0)) != cudaSuccess) return fail(e);
-    } else if (!same_layout) {
-        // inputs are ready, but the previous call's slots lie elsewhere: wait until it has finished with them
+    }
+    if (!same_layout) {
+        // the previous call on this device (from whatever stream) cut the workspace differently, or used another one that
+        // may overlap this one: its slots are not this call's slots, so the per-slot events do not protect them.  Wait
+        // until it has finished with all of them (a no-op when nothing is in flight).
         if ((e = cudaStreamWaitEvent(s->h2d, s->finish, 0)) != cudaSuccess) return fail(e);
     }
     s->last_workspace = workspace;

@@ -82,6 +82,10 @@ NFAD_DEV double rcp64_approx(double a)
 NFAD_DEV int double_hi(double a) { return __double2hiint(a); }
 NFAD_DEV int double_lo(double a) { return __double2loint(a); }
 NFAD_DEV double double_from(int hi, int lo) { return __hiloint2double(hi, lo); }
+// float -> double, exact (one conversion instruction on the special-function unit; forming the same bits with
+// integer operations was measured 6-15 % slower: these kernels have no issue slots to spare for it)
+NFAD_DEV double to_double(float x) { return double(x); }
+
 // double -> float, round to nearest even (subnormal results included)
 NFAD_DEV float to_float(double a) { return __double2float_rn(a); }
 

@@ -12,13 +12,10 @@ namespace nfad {
 template <class P> struct IsFast { static constexpr bool value = false; };
 template <> struct IsFast<Fast> { static constexpr bool value = true; };
 
-#ifndef NFAD_FWD16_UNROLL
-#define NFAD_FWD16_UNROLL 5
-#endif
 template <class K, class P> struct ForwardTrainOp {
     static constexpr int kMinBlocks = 0;
     // 16-bit storage: 5 packets per thread measured 1-4 % faster than 4 (3 and 6 are slower)
-    static constexpr int kUnroll = IsFast<P>::value ? NFAD_FWD16_UNROLL : 0;
+    static constexpr int kUnroll = IsFast<P>::value ? 5 : 0;
     static constexpr int kIn = 1, kOut = 2;
     static __device__ __forceinline__ constexpr bool keep(int k) { return k == 0; }   // y is consumed next; f' much later
     static __device__ __forceinline__ void apply(const float (&in)[1], float (&out)[2])
@@ -55,16 +52,10 @@ template <class K, class P> struct ForwardInferOp {
 //         sign), which the store's round-to-nearest-even takes to that zero (2^-134 itself is
 //         the tie between 0 and 2^-133, and 0 is the even one).
 // So there is no double rounding to repair and no data-dependent path in this kernel.
-#ifndef NFAD_BWD_MIN_BLOCKS
-#define NFAD_BWD_MIN_BLOCKS 4
-#endif
-#ifndef NFAD_BWD_UNROLL
-#define NFAD_BWD_UNROLL 0
-#endif
 struct BackwardOp {
     static constexpr int kIn = 2, kOut = 1;
-    static constexpr int kMinBlocks = NFAD_BWD_MIN_BLOCKS;   // measured: 4 is 7 % faster than 5 for this load-and-multiply kernel
-    static constexpr int kUnroll = NFAD_BWD_UNROLL;
+    static constexpr int kMinBlocks = 4;   // measured: 4 is 7 % faster than 5 for this load-and-multiply kernel
+    static constexpr int kUnroll = 0;
     static __device__ __forceinline__ constexpr bool keep(int) { return true; }
     static __device__ __forceinline__ void apply(const float (&in)[2], float (&out)[1]) { out[0] = __fmul_rn(in[0], in[1]); }
 };
@@ -108,7 +99,7 @@ template <> struct GateSlope<Swish> {
 template <> struct GateSlope<GeluTanh> {
     static __device__ __forceinline__ float of(float x, float h)
     {
-        float du2 = fmaf(0.2140747458f, x * x, 1.5957691216f);     // 2 sqrt(2/pi) (1 + 3 * 0.044715 x^2)
+        float du2 = fmaf(0.2140644488f, x * x, 1.5957691216f);     // 2 sqrt(2/pi) (1 + 3 * 0.044715 x^2)
         return du2 * (h * (1.0f - h));
     }
 };

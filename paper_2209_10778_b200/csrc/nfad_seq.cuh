@@ -64,10 +64,7 @@ __device__ __forceinline__ Dual<P> seq_apply(const SeqOp& o, const Dual<P>& a, c
 // Interprets the program for V elements, kSeqGroup at a time: the register file is indexed at
 // run time and so lives in local memory, and kSeqRegs x 2 x kSeqGroup scalars per thread is what
 // has to stay inside L1 for every resident thread.
-#ifndef NFAD_SEQ_GROUP
-#define NFAD_SEQ_GROUP 2
-#endif
-constexpr int kSeqGroup = NFAD_SEQ_GROUP;
+constexpr int kSeqGroup = 2;
 
 template <class P, int V>
 __device__ __forceinline__ void seq_run(const SeqProgram& prog, const float (&x)[V], float (&yv)[kSeqMaxOut][V],

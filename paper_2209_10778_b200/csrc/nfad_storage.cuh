@@ -18,24 +18,15 @@ namespace nfad {
 
 // Resident CTAs per SM the compiler must leave room for (a register cap).  The 16-bit kernels
 // are issue-bound with short dependency chains through MUFU: 5 CTAs (40 warps, <= 48 registers)
-// measured 3-5 % faster than the 4 the compiler picks by itself (7 or more spill and lose 30 %); the fp32 kernels need their
-// ~48 registers (a tighter cap spills).
-#ifndef NFAD_PDL
-#define NFAD_PDL 1
-#endif
-#ifndef NFAD_MIN_BLOCKS_16
-#define NFAD_MIN_BLOCKS_16 5
-#endif
-#ifndef NFAD_MIN_BLOCKS_32
-#define NFAD_MIN_BLOCKS_32 4
-#endif
+// measured 3-5 % faster than the 4 the compiler picks by itself (7 or more spill and lose 30 %); the fp32-storage kernels
+// hold their chains in double precision and need 64 registers (4 CTAs; a tighter cap spills, a looser one measured slower).
 
 // ---------------------------------------------------------------- storage types
 
 struct StoreF32 {
     using elem = float;
     static constexpr int kVec = 4;             // elements per 16-byte packet
-    static constexpr int kMinBlocks = NFAD_MIN_BLOCKS_32;
+    static constexpr int kMinBlocks = 4;
     static __device__ __forceinline__ void unpack(const uint4& p, float (&v)[4])
     {
         v[0] = __uint_as_float(p.x); v[1] = __uint_as_float(p.y);
@@ -52,7 +43,7 @@ struct StoreF32 {
 struct StoreBF16 {
     using elem = __nv_bfloat16;
     static constexpr int kVec = 8;
-    static constexpr int kMinBlocks = NFAD_MIN_BLOCKS_16;
+    static constexpr int kMinBlocks = 5;
     // a bf16 is the upper half of an fp32: widening is a shift or a mask
     static __device__ __forceinline__ void unpack(const uint4& p, float (&v)[8])
     {
@@ -79,7 +70,7 @@ struct StoreBF16 {
 struct StoreF16 {
     using elem = __half;
     static constexpr int kVec = 8;
-    static constexpr int kMinBlocks = NFAD_MIN_BLOCKS_16;
+    static constexpr int kMinBlocks = 5;
     static __device__ __forceinline__ void unpack(const uint4& p, float (&v)[8])
     {
         const uint32_t w[4] = {p.x, p.y, p.z, p.w};

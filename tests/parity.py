@@ -124,3 +124,21 @@ def full_check(kind: str, dtype: str, x: torch.Tensor, g: torch.Tensor, stats: d
         check_forward_16(kind, dtype, x_raw, y_raw, d_raw, stats)
     check_backward(dtype, g_raw, d_raw, gin_raw)
     return y, d, gin
+
+
+def recompute_backward_ok(kind: str, dtype: str, g_raw: np.ndarray, x_raw: np.ndarray, gin_raw: np.ndarray) -> np.ndarray:
+    """The recomputation comparator against the oracle's g f'(x), with the tolerance its arithmetic has and no more.
+    It forms g h + g x s(x, h) from the gate h ROUNDED to the storage type (unit roundoff u) and a slope s derived
+    from that rounded h by the operator's usual rule, then rounds once more:
+        |error| <= |g| ( u |h| (1 + |x| K) + 2^-20 (|h| + |x h'|) ) + u |g f'|
+    with K = max |ds/dh| (sigmoid: |1 - 2h| <= 1; the tanh form: that times 2 sqrt(2/pi) (1 + 3 a x^2); erf: the slope
+    does not use h, 0; tanh(softplus): 2 |t| sigmoid <= 2) and 2^-20 for the fp32 arithmetic of the rule itself.
+    |h| is bounded by |h| + |x h'|, which the oracle returns.  At small |x| this is a few roundings of g h: a wrong
+    constant in a slope rule fails it."""
+    f, fp, cond = oracle.forward(kind, dtype, x_raw, want_cond=True)
+    g, x, got = oracle.widen(dtype, g_raw), oracle.widen(dtype, x_raw), oracle.widen(dtype, gin_raw)
+    u = {"f32": 2.0 ** -24, "bf16": 2.0 ** -8, "f16": 2.0 ** -11}[dtype]      # half a unit in the last place
+    k = {"swish": 1.0, "gelu_erf": 0.0, "mish": 2.0, "gelu_tanh": 1.5957691216 * (1.0 + 0.134145 * x * x)}[kind]
+    tiny = {"f32": 2.0 ** -149, "bf16": 2.0 ** -133, "f16": 2.0 ** -24}[dtype]
+    tol = np.abs(g) * cond * (u * (1.0 + np.abs(x) * k) + 2.0 ** -20) + u * np.abs(g * fp) * 1.0001 + tiny
+    return np.abs(got - g * fp) <= tol

@@ -142,8 +142,8 @@ def test_conventional_comparator(kind, dtype):
 @pytest.mark.parametrize("kind", KINDS)
 @pytest.mark.parametrize("dtype", ["f32", "bf16", "f16"])
 def test_recompute_comparator(kind, dtype):
-    # operator-by-operator rules through a stored intermediate: the tolerance is the one that
-    # arithmetic has -- an absolute error of a few storage-type ulps of the gate, times |g| (1 + |x|)
+    # operator-by-operator rules through a stored intermediate: the tolerance is the one that arithmetic has
+    # (parity.recompute_backward_ok)
     n = (1 << 16) + 5
     x = W.draw("normal", n, dtype, 41, DEV)
     g = W.normal(n, dtype, 42, 1.0, DEV)
@@ -153,12 +153,8 @@ def test_recompute_comparator(kind, dtype):
     scratch = torch.empty(nbytes, dtype=torch.uint8, device=DEV)
     nfad.nfad_cmp_recompute_backward(kind, g, x, scratch, gin)
     torch.cuda.synchronize()
-    f, fp = oracle.forward(kind, dtype, W.raw_numpy(x))
-    gw, xw = oracle.widen(dtype, W.raw_numpy(g)), oracle.widen(dtype, W.raw_numpy(x))
-    got = oracle.widen(dtype, W.raw_numpy(gin))
-    eps = {"f32": 2.0 ** -23, "bf16": 2.0 ** -8, "f16": 2.0 ** -11}[dtype]
-    tol = np.abs(gw) * eps * (4 + 8 * np.abs(xw) * (1 + xw * xw / 4)) + eps * np.abs(gw * fp)
-    assert (np.abs(got - gw * fp) <= tol).all()
+    ok = parity.recompute_backward_ok(kind, dtype, W.raw_numpy(g), W.raw_numpy(x), W.raw_numpy(gin))
+    assert ok.all(), f"{(~ok).sum()} of {n} outside tolerance"
     with pytest.raises(nfad.NfadError) as e:
         nfad.nfad_cmp_recompute_backward(kind, g, x, scratch[:16], gin)
     assert e.value.status == 7

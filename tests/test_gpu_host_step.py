@@ -104,3 +104,29 @@ def test_host_step_inputs_ready_with_changing_workspaces():
         nfad.nfad_act_forward(kind, xd, yd, dd)
         nfad.nfad_act_backward(kind, gd, dd, gid)
         assert np.array_equal(W.raw_numpy(y), W.raw_numpy(yd)) and np.array_equal(W.raw_numpy(gi), W.raw_numpy(gid))
+
+
+def test_host_step_two_streams_sharing_one_workspace_with_different_cuts():
+    # two callers on different streams hand the SAME workspace to calls that cut it differently (other dtype and size,
+    # stream-ordered inputs): the second call must wait until the first has finished with its slots
+    n1, n2 = 6 * (1 << 20) + 77, 2 * (1 << 20) + 9
+    x1, g1 = W.normal(n1, "bf16", 81, 1.0).pin_memory(), W.normal(n1, "bf16", 82, 1.0).pin_memory()
+    x2, g2 = W.normal(n2, "f32", 83, 1.0).pin_memory(), W.normal(n2, "f32", 84, 1.0).pin_memory()
+    y1, gi1 = torch.empty_like(x1).pin_memory(), torch.empty_like(x1).pin_memory()
+    y2, gi2 = torch.empty_like(x2).pin_memory(), torch.empty_like(x2).pin_memory()
+    ws = torch.empty(nfad.nfad_host_step_workspace_bytes(torch.bfloat16, n1), dtype=torch.uint8, device=DEV)
+    sa, sb = torch.cuda.Stream(), torch.cuda.Stream()
+    torch.cuda.synchronize()
+    for _ in range(3):
+        with torch.cuda.stream(sa):
+            nfad.nfad_host_step("gelu_tanh", x1, g1, y1, None, gi1, ws)
+        with torch.cuda.stream(sb):
+            nfad.nfad_host_step("mish", x2, g2, y2, None, gi2, ws)
+    torch.cuda.synchronize()
+    for kind, x, g, y, gi in (("gelu_tanh", x1, g1, y1, gi1), ("mish", x2, g2, y2, gi2)):
+        xd, gd = x.to(DEV), g.to(DEV)
+        yd, dd, gid = torch.empty_like(xd), torch.empty_like(xd), torch.empty_like(xd)
+        nfad.nfad_act_forward(kind, xd, yd, dd)
+        nfad.nfad_act_backward(kind, gd, dd, gid)
+        torch.cuda.synchronize()
+        assert np.array_equal(W.raw_numpy(y), W.raw_numpy(yd)) and np.array_equal(W.raw_numpy(gi), W.raw_numpy(gid))

@@ -1,10 +1,14 @@
 """GPU tests of run-time FAD sequences: the fused executor and the operator-by-operator
 executor against the fp64 sequence oracle, the M-result backward, the autograd wrappers.
 
-Tolerance of this executor (plain fp32 primitives for every storage type, no hardening):
-  fp32     |got - o| <= 2e-5 * max(|o|, S) with S the size of the largest intermediate sum
-           feeding the result (taken as 1 + |x| here), i.e. a few fp32 ulp of the terms;
-  16-bit   within 1 ulp of the rounded oracle value, or within the fp32 tolerance above.
+Tolerances:
+  fp32     (double-precision primitives, one rounding at the store) |got - o| <= 8 ulp32(o), plus 2^-40 (1 + |x|)
+           of absolute slack for a derivative that passes through zero; inputs reach |x| = 20;
+  16-bit   (plain fp32 primitives) within 1 ulp of the rounded oracle value, or within 2e-5 * max(|o|, 1 + |x|):
+           a few fp32 ulp of the largest intermediate term feeding the result.
+A program that forms 1 + tanh(u) literally has the cancellation that expression has: it is held to these bounds where
+the expression is well conditioned, and a separate test shows that it loses digits in the tail while the fused
+primitive does not.
 """
 import numpy as np
 import pytest
@@ -40,14 +44,32 @@ PROGRAMS = {
 }
 
 
+FP32_SEQ_ULPS = 8.0
+
+
+def _as_passed(ops):
+    """The program as it crosses the boundary: its constants are fp32 there (nfad_seq_op.c is a float), so the oracle is
+    given those very constants, not the doubles they were written as."""
+    return [(o, a, b, d, float(np.float32(c))) for o, a, b, d, c in ops]
+
+
 def _close(dtype, got_t, want64, x64):
     got_raw = W.raw_numpy(got_t)
     got = oracle.widen(dtype, got_raw)
+    if dtype == "f32":
+        return np.abs(got - want64) <= FP32_SEQ_ULPS * ulp.ulp32(want64) + 2.0 ** -40 * (1.0 + np.abs(x64))
     tol32 = 2e-5 * np.maximum(np.abs(want64), 1.0 + np.abs(x64))
-    ok = np.abs(got - want64) <= tol32
-    if dtype != "f32":
-        ok |= ulp.ulp_distance16(got_raw, oracle.round_to(dtype, want64)) <= 1
-    return ok
+    return (np.abs(got - want64) <= tol32) | (ulp.ulp_distance16(got_raw, oracle.round_to(dtype, want64)) <= 1)
+
+
+def _inputs(name, dtype, n, seed):
+    """N(0, 4^2) clamped to |x| <= 20 for fp32 (16-bit: |x| <= 7, where plain fp32 primitives hold their bound); the
+    literal 1 + tanh program only where that sum is well conditioned."""
+    lim = 20.0 if dtype == "f32" else 7.0
+    x = W.normal(n, "f32", seed, 4.0 if dtype == "f32" else 2.0, DEV).clamp_(-lim, lim)
+    if name == "gelu_tanh_literal":
+        x = x.clamp_(min=-4.0)
+    return x.to(W.TORCH_DTYPES[dtype])
 
 
 @pytest.fixture(params=["interpreter", "compiled"])
@@ -74,7 +96,7 @@ def executor(request):
 def test_fused_executor_against_the_sequence_oracle(name, dtype, executor):
     prog = PROGRAMS[name]()
     n = 70001
-    x = (W.normal(n, "f32", 5, 2.0, DEV).clamp_(-7, 7)).to(W.TORCH_DTYPES[dtype])
+    x = _inputs(name, dtype, n, 5)
     try:
         ys, ds = sequence.run_fused(prog, x)
     except Exception:
@@ -83,7 +105,7 @@ def test_fused_executor_against_the_sequence_oracle(name, dtype, executor):
     torch.cuda.synchronize()
     assert nfad.nfad_seq_last_executor() == executor
     x64 = oracle.widen(dtype, W.raw_numpy(x))
-    y, d = oracle.seq_forward(prog.ops, x64, prog.n_out)
+    y, d = oracle.seq_forward(_as_passed(prog.ops), x64, prog.n_out)
     for k in range(prog.n_out):
         assert _close(dtype, ys[k], y[k], x64).all(), (name, dtype, "value", k)
         assert _close(dtype, ds[k], d[k], x64).all(), (name, dtype, "derivative", k)
@@ -121,7 +143,7 @@ def test_fused_executor_edges_and_unaligned(dtype, executor):
             nfad.nfad_seq_forward(prog.ops, x, [yb[off:off + n]], [db[off + 1:off + 1 + n]] if off == 3 else [db[off:off + n]])
             torch.cuda.synchronize()
             x64 = oracle.widen(dtype, W.raw_numpy(x))
-            y, d = oracle.seq_forward(prog.ops, x64, 1)
+            y, d = oracle.seq_forward(_as_passed(prog.ops), x64, 1)
             assert _close(dtype, yb[off:off + n], y[0], x64).all()
             assert (yb[:off] == 7.0).all() and (yb[off + n:] == 7.0).all()
             dsl = db[off + 1:off + 1 + n] if off == 3 else db[off:off + n]
@@ -156,12 +178,16 @@ def test_backward_of_a_two_result_sequence(dtype):
     assert np.array_equal(W.raw_numpy(one), W.raw_numpy(ref))
 
 
+@pytest.mark.parametrize("dtype", ["f32", "bf16", "f16"])
 @pytest.mark.parametrize("name", ["swish", "gelu_tanh", "mish", "two_results"])
-def test_operator_by_operator_executor(name):
-    dtype = "f32"
+def test_operator_by_operator_executor(name, dtype):
+    """One kernel per operator, every intermediate ROUNDED to the storage type on its way through memory: the bound is
+    a few storage-type roundings of the largest term, not the fused executor's."""
     prog = PROGRAMS[name]()
     n = 40009
-    x = W.normal(n, "f32", 9, 1.5, DEV).clamp_(-6, 6)
+    x = W.normal(n, "f32", 9, 1.5, DEV).clamp_(-6, 6).to(W.TORCH_DTYPES[dtype])
+    es = x.element_size()
+    eps = {"f32": 2.0 ** -24, "bf16": 2.0 ** -8, "f16": 2.0 ** -11}[dtype]       # half a unit in the last place
     ex = sequence.OpByOp(prog)
     outs = ex.forward(x)
     kept = ex.saved_bytes()
@@ -169,17 +195,19 @@ def test_operator_by_operator_executor(name):
     gin = ex.backward(gs)
     torch.cuda.synchronize()
     x64 = oracle.widen(dtype, W.raw_numpy(x))
-    y, d = oracle.seq_forward(prog.ops, x64, prog.n_out)
+    y, d = oracle.seq_forward(_as_passed(prog.ops), x64, prog.n_out)
+    ops_deep = 8.0                                           # roundings on the longest path of these programs
     for k in range(prog.n_out):
-        assert _close(dtype, outs[k], y[k], x64).all()
+        got = oracle.widen(dtype, W.raw_numpy(outs[k]))
+        assert (np.abs(got - y[k]) <= ops_deep * eps * np.maximum(np.abs(y[k]), 1.0 + np.abs(x64))).all(), (name, dtype, k)
     g64 = np.stack([oracle.widen(dtype, W.raw_numpy(g)) for g in gs])
     s, sa = oracle.seq_backward(g64, d)
     got = oracle.widen(dtype, W.raw_numpy(gin))
-    assert (np.abs(got - s) <= 4e-5 * np.maximum(sa, np.abs(g64).sum(0) * (1 + np.abs(x64)))).all()
+    assert (np.abs(got - s) <= 4 * ops_deep * eps * np.maximum(sa, np.abs(g64).sum(0) * (1 + np.abs(x64)))).all(), (name, dtype)
     # what operator-by-operator back-propagation keeps: Swish keeps x and sigmoid(x) (the paper's v1, v2)
     if name == "swish":
-        assert kept == 2 * n * 4
-    assert kept >= 2 * n * 4
+        assert kept == 2 * n * es
+    assert kept >= 2 * n * es
 
 
 def test_autograd_wrappers():
@@ -212,7 +240,7 @@ def test_autograd_wrappers():
     (a.sum() * 2.0 + b.sum()).backward()
     torch.cuda.synchronize()
     x64 = x.detach().double().cpu().numpy()
-    y, d = oracle.seq_forward(prog.ops, x64, 2)
+    y, d = oracle.seq_forward(_as_passed(prog.ops), x64, 2)
     want = 2.0 * d[0] + d[1]
     assert np.allclose(x.grad.double().cpu().numpy(), want, rtol=2e-5, atol=2e-5)
 
@@ -251,7 +279,7 @@ def test_four_results_forward_and_backward(dtype, executor):
     gin = sequence.backward_fused(gs, ds)
     torch.cuda.synchronize()
     x64 = oracle.widen(dtype, W.raw_numpy(xt))
-    y, d = oracle.seq_forward(p.ops, x64, 4)
+    y, d = oracle.seq_forward(_as_passed(p.ops), x64, 4)
     for k in range(4):
         assert _close(dtype, ys[k], y[k], x64).all(), ("value", k)
         assert _close(dtype, ds[k], d[k], x64).all(), ("derivative", k)
@@ -318,3 +346,24 @@ def test_large_sliced_views_use_the_whole_device(dtype, executor):
     assert nfad.nfad_seq_last_executor() == executor
     # the element-wise path over the whole grid costs a small multiple of the packet path, not the ~10^3 of one CTA
     assert ms_mixed < 40 * ms_ref, (ms_mixed, ms_ref)
+
+
+def test_literal_one_plus_tanh_loses_digits_where_the_fused_primitive_does_not(executor):
+    """Table I's GELU written with a literal 1 + tanh(u) against the same function with the fused (1 + tanh u)/2
+    primitive, in the negative tail where tanh(u) -> -1.  fp32 storage (double-precision primitives): both agree with
+    the oracle down to x = -4; from x = -6.5 on the literal sum has lost its digits (1 + tanh u < 2^-38, and the
+    rounding of tanh u is 2^-53) while the fused program still holds 8 ulp.  bf16 storage (fp32 primitives): the same
+    happens from x = -5 on, where 1 + tanh u is below the 2^-24 rounding of tanh u."""
+    lit, fused = sequence.gelu_tanh_literal_program(), sequence.gelu_tanh_program()
+    for dtype, lo, hi in (("f32", -9.0, -6.5), ("bf16", -7.0, -5.0)):
+        n = 20001
+        x = torch.linspace(lo, hi, n, device=DEV).to(W.TORCH_DTYPES[dtype])
+        x64 = oracle.widen(dtype, W.raw_numpy(x))
+        want, _ = oracle.seq_forward(_as_passed(fused.ops), x64, 1)
+        (yf,), _ = sequence.run_fused(fused, x)
+        (yl,), _ = sequence.run_fused(lit, x)
+        torch.cuda.synchronize()
+        assert _close(dtype, yf, want[0], x64).all()
+        rel = np.abs(oracle.widen(dtype, W.raw_numpy(yl)) - want[0]) / np.abs(want[0])
+        worst_allowed = 2.0 ** -20 if dtype == "f32" else 2.0 ** -7
+        assert np.median(rel) > worst_allowed, (dtype, float(np.median(rel)))

@@ -11,6 +11,7 @@ import numpy as np
 import pytest
 import torch
 
+import parity
 from paper_2209_10778_b200 import binding as nfad
 from paper_2209_10778_b200 import workloads as W
 
@@ -42,6 +43,8 @@ def test_two_calls_in_a_row_match_the_caller_scratch_entry_point(dtype):
         want = _reference(kind, g, x)
         torch.cuda.synchronize()
         assert np.array_equal(W.raw_numpy(out), W.raw_numpy(want)), kind
+        # and, like that entry point, what the oracle's g f'(x) allows for this arithmetic
+        assert parity.recompute_backward_ok(kind, dtype, W.raw_numpy(g), W.raw_numpy(x), W.raw_numpy(out)).all(), kind
 
 
 def test_in_place_gradient_and_size_limit():
