@@ -13,8 +13,10 @@
  *     elements of `dtype` (NFAD_F32: float; NFAD_BF16: bfloat16; NFAD_F16: IEEE
  *     half).  Tensor shape is irrelevant to an element-wise pass.  The caller
  *     owns all memory; the library allocates none and keeps no state between
- *     calls.  Arithmetic is fp32 for every storage type; results are rounded to
- *     nearest-even once, at the store.  Subnormals are kept (no flush to zero).
+ *     calls.  Arithmetic is fp32 for the 16-bit storage types and fp64 for fp32
+ *     storage (a few fp32 ulp of the exact result cannot be held by fp32
+ *     arithmetic itself); results are rounded to nearest-even once, at the store.
+ *     Subnormals are kept (no flush to zero).
  *   - Pointers need only the natural alignment of `dtype`.  When all tensors of
  *     a call share one offset modulo 16 bytes the 128-bit path is used (elements
  *     before the first and after the last whole 16-byte packet are handled one
@@ -103,13 +105,13 @@ NFAD_API int nfad_act_forward(int kind, int dtype, const void* x, void* y, void*
 /*
  * Forward pass with the derivative held to the LITERAL 4-ulp bound for every input (fp32 storage
  * only; any other dtype gives NFAD_E_DTYPE).  For x < 0, f' = h + x h' (Eq. 3 applied to f = x h) is
- * a difference of two terms of similar size that changes sign, so arithmetic good to an fp32 ulp of
- * the terms -- what nfad_act_forward guarantees there -- is not good to an fp32 ulp of f' near the
- * sign change.  This entry point forms the two terms for x < 0 in fp64 and rounds their difference
- * once: dfdx is within 4 fp32 ulp (in fact about one) of the exact f'(x) for every finite x, the
+ * a difference of two terms of similar size that changes sign, so arithmetic good to a fraction of an
+ * fp32 ulp of the TERMS -- what nfad_act_forward guarantees there (2^-29 of each) -- is not good to an
+ * fp32 ulp of f' within about 2^-8 of the terms' size of the sign change.  This entry point forms the
+ * two terms for x < 0 to full fp64 accuracy and rounds their difference once: dfdx is within 4 fp32 ulp (in fact about one) of the exact f'(x) for every finite x, the
  * neighbours of the sign change included; results below 2^-126 are rounded once to the subnormal
  * grid.  y, and dfdx for x >= 0, are bit-identical to nfad_act_forward.  Same pointer, aliasing and
- * stream rules.  Costs fp64 arithmetic on every element with x < 0 (see the measured rates).
+ * stream rules.  Costs library-grade fp64 exponentials on every element with x < 0 (see the measured rates).
  * The 16-bit storage types need no such variant: there nfad_act_forward is within one ulp of the
  * correctly rounded f' for every input.
  */
@@ -225,9 +227,11 @@ NFAD_API int nfad_saved_bytes_per_element(int kind, int dtype, int layout);
  *   y, dfdx [host arrays of m device pointers, m <= 4] y[k][i] = k-th result, dfdx[k][i] its
  *           derivative with respect to x[i]: per result, the one tensor to keep.
  * One kernel runs the whole sequence per element on dual numbers; no intermediate reaches
- * memory.  Arithmetic: plain fp32 primitives for every storage type (a few fp32 ulp where
- * the composed function is well conditioned) -- the four activations of Table I have
- * dedicated, hardened entry points above.  Outputs must not overlap each other or x.
+ * memory.  Arithmetic: fp32 primitives for the 16-bit storage types (a few fp32 ulp where the
+ * composed function is well conditioned), fp64 primitives good to 2^-45 for fp32 storage (results
+ * within a few fp32 ulp of the exact ones wherever the program itself does not cancel).  The
+ * constants of a program are fp32 (`c` below).  The four activations of Table I have dedicated
+ * entry points above.  Outputs must not overlap each other or x.
  */
 typedef enum {
     NFAD_OP_ADD = 0, NFAD_OP_MUL = 1, NFAD_OP_SCALE = 2, NFAD_OP_ADD_CONST = 3, NFAD_OP_EXP = 4, NFAD_OP_LOG1P = 5,

@@ -14,8 +14,10 @@ template <> struct IsFast<Fast> { static constexpr bool value = true; };
 
 template <class K, class P> struct ForwardTrainOp {
     static constexpr int kMinBlocks = 0;
-    // 16-bit storage: 5 packets per thread measured 1-4 % faster than 4 (3 and 6 are slower)
-    static constexpr int kUnroll = IsFast<P>::value ? 5 : 0;
+    // packets per thread and tile, measured at 100.7M elements: 16-bit storage 5 (1-4 % faster than 4; 3 and 6 are slower
+    // under the 48-register cap), fp32 storage 7 (0.76 / 0.82 / 0.95 / 0.87 of the copy peak against 0.72 / 0.82 / 0.88 /
+    // 0.84 with 4; 8 and 10 fall off again)
+    static constexpr int kUnroll = IsFast<P>::value ? 5 : 7;
     static constexpr int kIn = 1, kOut = 2;
     static __device__ __forceinline__ constexpr bool keep(int k) { return k == 0; }   // y is consumed next; f' much later
     static __device__ __forceinline__ void apply(const float (&in)[1], float (&out)[2])
@@ -29,7 +31,9 @@ template <class K, class P> struct ForwardTrainOp {
 // Forward, inference: x -> y.  Same chain; the tangent parts are dead code.
 template <class K, class P> struct ForwardInferOp {
     static constexpr int kMinBlocks = 0;
-    static constexpr int kUnroll = 0;
+    // one input stream and one output: six packets per thread (16-bit storage) and eight (fp32 storage) measured 5-10 %
+    // faster than four
+    static constexpr int kUnroll = IsFast<P>::value ? 6 : 8;
     static constexpr int kIn = 1, kOut = 1;
     static __device__ __forceinline__ constexpr bool keep(int) { return true; }
     static __device__ __forceinline__ void apply(const float (&in)[1], float (&out)[1])
@@ -63,10 +67,11 @@ struct BackwardOp {
 // Conventional layout: x is saved, and backward re-derives f'(x) with the full
 // transcendental chain before the multiply.
 template <class K, class P> struct ConvBackwardOp {
-    // two input streams of four packets each are 32 registers before any arithmetic: room for 64 (four resident CTAs),
-    // or the chain's temporaries spill
+    // two input streams: their packets alone are 24-40 registers, so room for 64 (four resident CTAs) or the chain's
+    // temporaries spill.  Packets per thread, measured at 100.7M elements: 16-bit storage 5 (0.90-1.02 of the copy peak
+    // against 0.80-0.89 with 4), fp32 storage 3 (0.72-0.91 against 0.70-0.87)
     static constexpr int kMinBlocks = 4;
-    static constexpr int kUnroll = 0;
+    static constexpr int kUnroll = IsFast<P>::value ? 5 : 3;
     static constexpr int kIn = 2, kOut = 1;
     static __device__ __forceinline__ constexpr bool keep(int) { return true; }
     static __device__ __forceinline__ void apply(const float (&in)[2], float (&out)[1])
@@ -81,7 +86,7 @@ template <class K, class P> struct ConvBackwardOp {
 // walks those rules: x' = g v1 + g v2 v1' with v2 = x (Eq. 2).
 template <class K, class P> struct RecomputePhase1Op {
     static constexpr int kMinBlocks = 0;
-    static constexpr int kUnroll = 0;
+    static constexpr int kUnroll = IsFast<P>::value ? 6 : 8;      // the same shape as the value-only forward
     static constexpr int kIn = 1, kOut = 1;
     static __device__ __forceinline__ constexpr bool keep(int) { return true; }
     static __device__ __forceinline__ void apply(const float (&in)[1], float (&out)[1])
