@@ -107,13 +107,14 @@ NFAD_API int nfad_act_forward(int kind, int dtype, const void* x, void* y, void*
  * only; any other dtype gives NFAD_E_DTYPE).  For x < 0, f' = h + x h' (Eq. 3 applied to f = x h) is
  * a difference of two terms of similar size that changes sign, so arithmetic good to a fraction of an
  * fp32 ulp of the TERMS -- what nfad_act_forward guarantees there (2^-29 of each) -- is not good to an
- * fp32 ulp of f' within about 2^-8 of the terms' size of the sign change.  This entry point forms the
- * two terms for x < 0 to full fp64 accuracy and rounds their difference once: dfdx is within 4 fp32 ulp (in fact about one) of the exact f'(x) for every finite x, the
- * neighbours of the sign change included; results below 2^-126 are rounded once to the subnormal
- * grid.  y, and dfdx for x >= 0, are bit-identical to nfad_act_forward.  Same pointer, aliasing and
- * stream rules.  Costs library-grade fp64 exponentials on every element with x < 0 (see the measured rates).
- * The 16-bit storage types need no such variant: there nfad_act_forward is within one ulp of the
- * correctly rounded f' for every input.
+ * fp32 ulp of f' within about 2^-8 of the terms' size of the sign change.  This entry point runs the
+ * same dual-number chain on primitives good to the last bits of a double and rounds once: y and dfdx
+ * are within about one fp32 ulp of the exact f(x) and f'(x) for every finite x, the fp32 neighbours of
+ * the sign change included; results below 2^-126 are rounded once to the subnormal grid.  Away from
+ * the sign change it agrees with nfad_act_forward to the last place or the one before.  Same pointer,
+ * aliasing and stream rules.  Costs about twice the fp64 arithmetic of nfad_act_forward (see the
+ * measured rates).  The 16-bit storage types need no such variant: there nfad_act_forward is within
+ * one ulp of the correctly rounded f' for every input.
  */
 NFAD_API int nfad_act_forward_strict(int kind, int dtype, const void* x, void* y, void* dfdx, size_t n, nfad_stream_t stream);
 

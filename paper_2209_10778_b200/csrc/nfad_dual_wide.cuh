@@ -212,18 +212,22 @@ NFAD_DEV Gate<Wide> dual_half_one_plus_erf_scaled(Wide, double c, const Seed& a)
 // ----------------------------------------------------------------- softplus, and tanh of a softplus
 
 // softplus remembers w = exp(v) itself: its slope sigmoid(v) and tanh(softplus) are algebraic in w
+// (tag Precise: the exponential and the reciprocal to 2^-52 instead of 2^-29, as in the general-purpose primitives)
+struct Precise {};
 template <> struct SoftplusDual<Wide> { double w; };
 NFAD_DEV SoftplusDual<Wide> dual_softplus(Wide, const Seed& a) { return {wide::exp_bounded<6>(hw::to_double(a.x))}; }
+NFAD_DEV SoftplusDual<Wide> dual_softplus(Wide, Precise, const Seed& a) { return {wide::exp_bounded<11>(hw::to_double(a.x))}; }
 
 // one form for both signs, every term positive:  T = n/(n + 2),  n = w (w + 2),  w = e^v;
 // T' = (dn/dv) 2/(n + 2)^2 = 4 w (w + 1)/(n + 2)^2.  |v| <= 150 keeps (n + 2)^2 inside the range of a double.
-NFAD_DEV Gate<Wide> dual_tanh(const SoftplusDual<Wide>& p)
+template <int kRcpSteps> NFAD_DEV Gate<Wide> tanh_of_softplus_wide(double w)
 {
-    double w = p.w;
     double n = w * (w + 2.0);
-    double rd = wide::rcp<1>(n + 2.0);
+    double rd = wide::rcp<kRcpSteps>(n + 2.0);
     return {n * rd, (4.0 * (w * rd)) * ((w + 1.0) * rd)};
 }
+NFAD_DEV Gate<Wide> dual_tanh(const SoftplusDual<Wide>& p) { return tanh_of_softplus_wide<1>(p.w); }
+NFAD_DEV Gate<Wide> dual_tanh(Precise, const SoftplusDual<Wide>& p) { return tanh_of_softplus_wide<2>(p.w); }
 
 // ----------------------------------------------------------------- general-purpose primitives
 //

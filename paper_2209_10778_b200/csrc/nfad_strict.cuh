@@ -1,75 +1,45 @@
-// nfad_strict.cuh -- f'(x) for x < 0 to a fraction of an fp32 ulp of f'(x) ITSELF.
+// nfad_strict.cuh -- f'(x) to a fraction of an fp32 ulp of f'(x) ITSELF, for every x.
 //
 // For x < 0 the derivative f' = h + x h' is the difference of two positive quantities A = h and
 // B = -x h' of similar size, and it changes sign (near -0.75 for the GELUs, -1.28 for Swish, -1.19
-// for Mish).  Arithmetic that is good to an fp32 ulp of A and B -- all that fp32 internals can give,
-// and what the regular forward pass guarantees -- is therefore not good to an fp32 ulp of A - B.
-// The strict forward pass evaluates A and B for x < 0 in fp64 (cancellation-free forms: every
-// exponential has a non-positive argument, 1 - sigmoid is formed as 1/(1+e), Phi as erfc/2) and
-// rounds the difference once: the result is within 0.5 ulp + 2^-52 (A + B)/|A - B| ulp... i.e. within
-// one fp32 ulp unless |f'| < 2^-27 (A + B), which no fp32 x reaches by more than a factor of two.
-// Results below 2^-126 are rounded once to the subnormal grid by the conversion itself.
+// for Mish).  The regular forward pass evaluates A and B to 2^-29 of themselves -- a thirtieth of an
+// fp32 ulp of the TERMS, which is what its tolerance asks for -- and that is not an fp32 ulp of
+// A - B within about 2^-8 (A + B) of the sign change.  The strict pass runs the same dual-number
+// chain (Section II-C approach 3, Eq. 3) on the general-purpose double-precision primitives, whose
+// exponential, reciprocal and erfc are good to the last bits of a double: the error of f' is then
+// 0.5 ulp + about 2^-27 (A + B)/|A - B| fp32 ulp, i.e. within one ulp even for the fp32 inputs
+// nearest to the sign change (no fp32 x brings |f'| below 2^-28 (A + B)).  Results below 2^-126
+// are rounded once to the subnormal grid by the conversion itself.
 #pragma once
 
 #include "nfad_dual.cuh"
 
 namespace nfad {
 
-// The argument is already clamped to [-kWide, 0): all exponentials stay finite and non-zero where it matters.
-__device__ __forceinline__ double fprime_negative_f64(GeluErf, double x)
+// The gate h(x) of each activation on the precise primitives (the argument is already clamped to the
+// activation's saturation range).
+NFAD_DEV Gate<Wide> gate_precise(GeluErf, Seed X) { return dual_half_one_plus_erf(dual_scale(Wide{}, 0.7071067811865476, X)); }
+NFAD_DEV Gate<Wide> gate_precise(GeluTanh, Seed X)
 {
-    const double kInvSqrt2 = 0.70710678118654752440, kInvSqrt2Pi = 0.39894228040143267794;
-    double a = 0.5 * erfc(-x * kInvSqrt2);                    // Phi(x)
-    double b = -x * (exp(-0.5 * x * x) * kInvSqrt2Pi);        // -x phi(x)
-    return a - b;
+    return dual_half_one_plus_tanh(dual_odd_cubic(Wide{}, 0.7978845608028654, 0.035677408136300125, 0.10703222440890037, X));
 }
+NFAD_DEV Gate<Wide> gate_precise(Swish, Seed X) { return dual_sigmoid(as_wide(X)); }
+NFAD_DEV Gate<Wide> gate_precise(Mish, Seed X) { return dual_tanh(Precise{}, dual_softplus(Wide{}, Precise{}, X)); }
 
-__device__ __forceinline__ double fprime_negative_f64(GeluTanh, double x)
+// x -> (f(x), f'(x))
+template <class K> NFAD_DEV ActOut evaluate_strict(float x)
 {
-    const double c = 0.79788456080286535588, a = 0.044715;
-    double x2 = x * x;
-    double u = c * (x + a * (x2 * x));                        // < 0
-    double e = exp(2.0 * u);
-    double big = 1.0 / (1.0 + e);                             // 1 - S
-    double s = e * big;                                       // S = (1 + tanh u)/2
-    double du2 = 2.0 * c * (1.0 + 3.0 * a * x2);              // 2 u'
-    return s - (-x * du2) * (s * big);
-}
-
-__device__ __forceinline__ double fprime_negative_f64(Swish, double x)
-{
-    double e = exp(x);
-    double big = 1.0 / (1.0 + e);
-    double s = e * big;
-    return s - (-x) * (s * big);
-}
-
-__device__ __forceinline__ double fprime_negative_f64(Mish, double x)
-{
-    double w = exp(x);
-    double n = w * (w + 2.0);
-    double den = n + 2.0;
-    double t = n / den;                                       // tanh(softplus x)
-    double sech2 = 4.0 * (n + 1.0) / (den * den);
-    double sig = w / (1.0 + w);
-    return t - (-x) * (sech2 * sig);
-}
-
-// x -> (f(x), f'(x)): the value and, for x >= 0, the derivative from the regular fp32-storage chain
-// (within a rounding of themselves there); the derivative for x < 0 from the forms above.
-template <class K> __device__ __forceinline__ ActOut evaluate_strict(float x)
-{
-    ActOut o = evaluate(K{}, Wide{}, x);
-    if (x < 0.0f) {
-        constexpr float kSat = Saturation<K>::kWide;
-        o.dydx = __double2float_rn(fprime_negative_f64(K{}, (double)fmaxf(x, -kSat)));
-    }
-    return o;
+    constexpr float kSat = Saturation<K>::kWide;
+    float xc = hw::clamp_nan(x, -kSat, kSat);
+    Seed X{xc};
+    Gate<Wide> Y = dual_mul(X, gate_precise(K{}, X));
+    float y = dual_value(Y);
+    return {x > kSat ? x : y, dual_tangent(Y)};
 }
 
 template <class K> struct ForwardStrictOp {
-    static constexpr int kMinBlocks = 3;
-    static constexpr int kUnroll = 2;
+    static constexpr int kMinBlocks = 0;
+    static constexpr int kUnroll = 4;
     static constexpr int kIn = 1, kOut = 2;
     static __device__ __forceinline__ constexpr bool keep(int k) { return k == 0; }
     static __device__ __forceinline__ void apply(const float (&in)[1], float (&out)[2])

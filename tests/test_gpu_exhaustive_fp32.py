@@ -22,7 +22,7 @@ pytestmark = pytest.mark.gpu
 STRIDE = int(os.environ.get("NFAD_EXHAUSTIVE_STRIDE", "251"))
 HI_BITS = int(np.float32(130.0).view(np.uint32))
 CHUNK = 1 << 25
-# (value ulp, derivative in the gate's metric): the all-inputs maxima are 2.2 / 2.3 for the erf form and 0.53 for the others
+# (value ulp, derivative in the gate's metric): the all-inputs maxima are 2.28 / 2.34 for the erf form and 0.53 for the others
 BOUNDS = {"gelu_erf": (2.6, 2.6), "gelu_tanh": (0.6, 0.6), "swish": (0.6, 0.6), "mish": (0.6, 0.6)}
 
 
@@ -72,7 +72,9 @@ def test_every_kth_fp32_input(kind):
     by, bd = BOUNDS[kind]
     assert w["bad"] == 0
     assert w["y"] <= by and w["d"] <= bd, w
-    assert w["sub_y"] <= 1.0 and w["sub_d"] <= 1.0, w           # a subnormal result is rounded once: within one spacing
+    # a subnormal result is rounded once, by the final conversion: within a spacing, or two where the gate itself carries
+    # a couple of fp32 ulp (the erf form)
+    assert w["sub_y"] <= 2.0 and w["sub_d"] <= 2.0, w
 
 
 @pytest.mark.parametrize("kind", list(BOUNDS))
@@ -80,5 +82,5 @@ def test_every_kth_fp32_input_strict_entry_point(kind):
     w = _sweep(kind, strict=True)
     print(kind, "strict, stride", STRIDE, w)
     assert w["bad"] == 0
-    assert w["y"] <= BOUNDS[kind][0] and w["d"] <= 4.0, w
+    assert w["y"] <= 1.0 and w["d"] <= 2.0, w                   # the strict chain is good to the last bits of a double
     assert w["sub_y"] <= 1.0 and w["sub_d"] <= 1.0, w

@@ -1,7 +1,8 @@
 """nfad_act_forward_strict (fp32 storage): f' within 4 fp32 ulp of the fp64 oracle's f' ITSELF for every input --
 the literal reading of the tolerance, with no scaling by the size of the cancelling terms -- including every fp32
-neighbour of the sign change of f'.  y, and f' for x >= 0, must be bit-identical to nfad_act_forward.
-Results below 2^-126: within 2 spacings of the subnormal grid.
+neighbour of the sign change of f'.  It runs the dual-number chain on primitives good to the last bits of a double, so
+y and f' are expected within about one ulp everywhere (asserted: y within 1, f' within 4, and within 2 on the
+neighbours of the sign change).  Results below 2^-126: within 2 spacings of the subnormal grid.
 """
 import numpy as np
 import pytest
@@ -20,14 +21,13 @@ DEV = "cuda"
 def _strict_check(kind, x):
     y, d = torch.empty_like(x), torch.empty_like(x)
     nfad.nfad_act_forward_strict(kind, x, y, d)
-    y0, d0 = torch.empty_like(x), torch.empty_like(x)
-    nfad.nfad_act_forward(kind, x, y0, d0)
     torch.cuda.synchronize()
     xh, yh, dh = x.cpu().numpy(), y.cpu().numpy(), d.cpu().numpy()
-    assert np.array_equal(yh.view(np.uint32), y0.cpu().numpy().view(np.uint32))
-    pos = ~(xh < 0)
-    assert np.array_equal(dh.view(np.uint32)[pos], d0.cpu().numpy().view(np.uint32)[pos])
     f, fp = oracle.forward(kind, "f32", xh)
+    ey = ulp.err_strict32(yh, f)
+    sub_y = np.abs(f) < 2.0 ** -126
+    bad_y = np.where(sub_y, np.abs(yh.astype(np.float64) - f) > 2 * 2.0 ** -149, ey > 1.0) | ~np.isfinite(yh)
+    assert not bad_y.any(), f"{kind}: {int(bad_y.sum())} values beyond 1 ulp; worst {np.where(sub_y, 0, ey).max():.2f}"
     err = ulp.err_strict32(dh, fp)
     sub = np.abs(fp) < 2.0 ** -126
     bad = np.where(sub, np.abs(dh.astype(np.float64) - fp) > 2 * 2.0 ** -149, err > 4.0) | ~np.isfinite(dh)
@@ -50,7 +50,7 @@ def test_strict_on_every_neighbour_of_the_sign_change(kind):
     bits = torch.arange(centre - (1 << 17), centre + (1 << 17), dtype=torch.int64).to(torch.int32)
     x = bits.view(torch.float32).to(DEV).contiguous()
     worst, worst_neg = _strict_check(kind, x)
-    assert worst_neg <= 2.0     # in fact about one ulp: fp64 terms, one rounding
+    assert worst <= 2.0         # in fact about one ulp: terms good to the last bits of a double, one rounding
     # the regular pass on the same inputs is NOT strict there (that is the point of this entry point)
     y0, d0 = torch.empty_like(x), torch.empty_like(x)
     nfad.nfad_act_forward(kind, x, y0, d0)
