@@ -22,9 +22,11 @@
 //     dual_half_one_plus_erf_scaled(c, x) = (1 + erf(c x))/2 of the seed
 //     dual_odd_cubic(c1, c3, x)         = c1 x + c3 x^3,  tangent c1 + 3 c3 x^2
 //
-// Policies.  Fast (16-bit storage, this file): a value and a tangent are one float each, on
-// the hardware's approximate exponential and reciprocal.  Wide (fp32 storage,
-// nfad_dual_wide.cuh): the same algebra in double precision.
+// Policies.  Fast (16-bit storage): a value and a tangent are one float each, on the hardware's
+// approximate exponential and reciprocal; this file holds its general-purpose primitives (for
+// sequences composed at run time), nfad_dual_fast.cuh the chains of the four activations, written
+// once for one element per call (Fast) and for two on packed fp32 arithmetic (Fast2).  Wide (fp32
+// storage, nfad_dual_wide.cuh): the same algebra in double precision.
 //
 // Gates.  sigmoid, (1+tanh)/2, (1+erf)/2 and tanh(softplus) are the factors h(x) of the four
 // activations f(x) = x h(x); a `Gate` is the dual number (h, h').
@@ -61,59 +63,35 @@ NFAD_DEV Dual<Fast> dual_add(const Dual<Fast>& a, const Dual<Fast>& b) { return 
 // c + a (binary with one constant input: unary, tangent unchanged)
 NFAD_DEV Dual<Fast> dual_add_const(float c, const Dual<Fast>& a) { return {c + a.v, a.t}; }
 
-// c * a   (a seed does not say which policy its result takes: the caller passes it as a tag)
+// c * a
 NFAD_DEV Dual<Fast> dual_scale(float c, const Dual<Fast>& a) { return {c * a.v, c * a.t}; }
-NFAD_DEV Dual<Fast> dual_scale(Fast, float c, const Seed& a) { return {c * a.x, c}; }
 
 // ----------------------------------------------------------------- mul (product rule, Eq. 3)
-
-NFAD_DEV Dual<Fast> dual_mul(Fast, const Seed& a, const Seed& b) { return {a.x * b.x, a.x + b.x}; }
-
-// x * b:  value x b.v,  tangent 1 * b.v + x * b.t
-NFAD_DEV Dual<Fast> dual_mul(const Seed& a, const Dual<Fast>& b) { return {a.x * b.v, fmaf(a.x, b.t, b.v)}; }
-NFAD_DEV Gate<Fast> dual_mul(const Seed& a, const Gate<Fast>& b) { return {a.x * b.v, fmaf(a.x, b.t, b.v)}; }
 
 NFAD_DEV Dual<Fast> dual_mul(const Dual<Fast>& a, const Dual<Fast>& b)
 {
     return {a.v * b.v, fmaf(a.v, b.t, a.t * b.v)};
 }
 
-// ----------------------------------------------------------------- odd cubic of the seed
-
-// p(x) = c1 x + c3 x^3 = x (c1 + c3 x^2),  p'(x) = c1 + 3 c3 x^2   (k3 = 3 c3 is passed in).
-NFAD_DEV Dual<Fast> dual_odd_cubic(Fast, float c1, float c3, float k3, const Seed& a)
-{
-    float s = a.x * a.x;
-    return {a.x * fmaf(c3, s, c1), fmaf(k3, s, c1)};
-}
-
 // ----------------------------------------------------------------- the logistic function and its slope
 
 // L(w) = 1/(1+exp(-w)), L' = L (1 - L), one form for both signs.  E = 2^-64 exp(-w) comes from one exponential on
-// the argument lowered by 64 (finite up to w = -133, and flushed to zero only where exp(-w) < 2^-62, far below what
-// a 16-bit result keeps); r = 1/(E + 2^-64);  L = 2^-64 r  and  1 - L = E r, with no subtraction anywhere, so both
-// tails keep their relative accuracy.  Needs scale * w >= -133 for the slope (E r would be inf * 0 beyond): kInRange
-// says that the caller has seen to that (the activations clamp x itself); otherwise the argument is clamped here.
+// the argument lowered by 64 (flushed to zero only where exp(-w) < 2^-62, far below what a 16-bit result keeps, and
+// clamped where it would overflow: beyond w = -133 the slope's E r would be inf * 0); r = 1/(E + 2^-64);
+// L = 2^-64 r  and  1 - L = E r, with no subtraction anywhere, so both tails keep their relative accuracy.
 // The slope is returned times slope_in * slope_const (the chain rule's next factor and a compile-time constant).
-template <bool kInRange>
 NFAD_DEV Gate<Fast> logistic_fast(float w, float minus_log2e_scale, float slope_in, float slope_const)
 {
-    float t = fmaf(w, minus_log2e_scale, -64.0f);
-    if (!kInRange) t = hw::min_nan(t, 126.0f);
-    float E = hw::ex2_approx_ftz(t);
+    float E = hw::ex2_approx_ftz(hw::min_nan(fmaf(w, minus_log2e_scale, -64.0f), 126.0f));
     float r = hw::rcp_approx(E + kTwoPowMinus64);
     float L = r * kTwoPowMinus64;
     return {L, (L * (E * r)) * (slope_in * slope_const)};
 }
 
-// sigmoid
-NFAD_DEV Gate<Fast> dual_sigmoid(Fast, const Seed& a) { return logistic_fast<false>(a.x, -1.44269502f, 1.0f, 1.0f); }
-NFAD_DEV Gate<Fast> dual_sigmoid(Fast, InRange, const Seed& a) { return logistic_fast<true>(a.x, -1.44269502f, 1.0f, 1.0f); }
-NFAD_DEV Gate<Fast> dual_sigmoid(const Dual<Fast>& a) { return logistic_fast<false>(a.v, -1.44269502f, a.t, 1.0f); }
+NFAD_DEV Gate<Fast> dual_sigmoid(const Dual<Fast>& a) { return logistic_fast(a.v, -1.44269502f, a.t, 1.0f); }
 
 // H = (1 + tanh u)/2 = L(2u),  dH/du = 2 L'(2u)   [= (1 - tanh^2 u)/2]
-NFAD_DEV Gate<Fast> dual_half_one_plus_tanh(const Dual<Fast>& u) { return logistic_fast<false>(u.v, -2.88539004f, u.t, 2.0f); }
-NFAD_DEV Gate<Fast> dual_half_one_plus_tanh(InRange, const Dual<Fast>& u) { return logistic_fast<true>(u.v, -2.88539004f, u.t, 2.0f); }
+NFAD_DEV Gate<Fast> dual_half_one_plus_tanh(const Dual<Fast>& u) { return logistic_fast(u.v, -2.88539004f, u.t, 2.0f); }
 
 // ----------------------------------------------------------------- (1 + erf z)/2
 
@@ -129,44 +107,9 @@ NFAD_DEV Gate<Fast> dual_half_one_plus_erf(const Dual<Fast>& z)
     float a = e64 * half_erfcx_fast_scaled<6>(hw::rcp_approx(za + kErfcxShift));
     return {z.v < 0.0f ? a : 1.0f - a, e64 * (kInvSqrtPiScaled * z.t)};
 }
-// (1 + erf(c x))/2 of the seed, c a constant: the scale folded in (a binary operation with one constant input is
-// unary, Section III-A), which lets c^2 join the exponent's constant and c x + k be one fused multiply-add.
-// kDegree 6 for value and slope; 4 for the value alone (a pass that will not be differentiated): a 16-bit result
-// needs 2^-12 of the gate, not the 2^-16 that the cancelling combination in the derivative needs.
-template <int kDegree> NFAD_DEV Gate<Fast> dual_half_one_plus_erf_scaled(Fast, float c, const Seed& x)
-{
-    const float kInvSqrtPiScaled = 0.564189612865448f * 5.42101086e-20f;
-    float xa = fabsf(x.x);
-    float e64 = exp2_fast_times_2p64(fmaf(xa * xa, (c * c) * -1.44269502f, 64.0f));
-    float a = e64 * half_erfcx_fast_scaled<kDegree>(hw::rcp_approx(fmaf(xa, c, kErfcxShift)));
-    return {x.x < 0.0f ? a : 1.0f - a, e64 * (kInvSqrtPiScaled * c)};
-}
+// ----------------------------------------------------------------- softplus
 
-// ----------------------------------------------------------------- softplus, and tanh of a softplus
-
-// p = softplus(v) = log1p(exp v),  p' = sigmoid(v).
-// The result remembers w = exp(v): every later use of p in the Mish chain (its tangent, tanh p) is an algebraic
-// function of w, so the logarithm itself is never needed there.
-template <class P> struct SoftplusDual;
-template <> struct SoftplusDual<Fast> { float w; };
-
-// (v <= 20 by the caller's clamp.)  w is formed as 2^-64 (2^64 w) so that a result below 2^-126 is rounded by the
-// multiplier and not flushed by the exponential unit.
-NFAD_DEV SoftplusDual<Fast> dual_softplus(Fast, const Seed& a)
-{
-    return {exp2_fast_times_2p64(fmaf(a.x, 1.44269502f, 64.0f)) * kTwoPowMinus64};
-}
-
-// tanh(log1p(w)) = ((1+w)^2 - 1)/((1+w)^2 + 1) = n/(n + 2), n = w (w + 2): one form for both signs, every term
-// positive.  T' = (dn/dv) 2/(n + 2)^2 = 4 w (w + 1)/(n + 2)^2.  Needs w <= 2^29 (v <= 20), so that the factors of
-// the slope stay inside fp32's range.
-NFAD_DEV Gate<Fast> dual_tanh(const SoftplusDual<Fast>& p)
-{
-    float w = p.w;
-    float n = w * (w + 2.0f);
-    float rd = hw::rcp_approx(n + 2.0f);
-    return {n * rd, (4.0f * (w * rd)) * ((w + 1.0f) * rd)};
-}
+template <class P> struct SoftplusDual;        // what softplus hands to tanh in the Mish chain (nfad_dual_fast.cuh, nfad_dual_wide.cuh)
 
 // ----------------------------------------------------------------- general-purpose primitives
 //
@@ -231,6 +174,7 @@ NFAD_DEV Dual<Fast> dual_softplus(const Dual<Fast>& a)
 
 }  // namespace nfad
 
+#include "nfad_dual_fast.cuh"
 #include "nfad_dual_wide.cuh"
 
 namespace nfad {
@@ -265,18 +209,18 @@ template <> struct Saturation<Mish> {                    // tanh(softplus) is fo
     static constexpr float kFastGateLo = -3.40282347e+38f, kFastGateHi = 20.0f;
 };
 
-// The gate h(x) of each activation f(x) = x h(x), as a dual number.  The argument is inside the range that
-// Saturation states, so the primitives run without clamps of their own.
+// The gate h(x) of each activation f(x) = x h(x), as a dual number (per lane under Fast / Fast2).  The argument is
+// inside the range that Saturation states, so the primitives run without clamps of their own.
 
 // GELU, erf form: h = Phi(x) = (1 + erf(x/sqrt2))/2
-NFAD_DEV Gate<Fast> gate(Fast, GeluErf, Seed X) { return dual_half_one_plus_erf_scaled<6>(Fast{}, 0.707106769f, X); }
+template <class P> NFAD_DEV Gate<P> gate(P, GeluErf, SeedOf<P> X) { return dual_half_one_plus_erf_scaled<6>(P{}, 0.707106769f, X); }
 NFAD_DEV Gate<Wide> gate(Wide, GeluErf, Seed X) { return dual_half_one_plus_erf_scaled(Wide{}, 0.7071067811865476, X); }
 
 // GELU, tanh form (Table I): h = (1 + tanh(sqrt(2/pi) (x + 0.044715 x^3)))/2
 //   u = c x + (c a) x^3 with c = sqrt(2/pi), a = 0.044715 (the double nearest to it); the last constant is 3 c a
-NFAD_DEV Gate<Fast> gate(Fast, GeluTanh, Seed X)
+template <class P> NFAD_DEV Gate<P> gate(P, GeluTanh, SeedOf<P> X)
 {
-    return dual_half_one_plus_tanh(InRange{}, dual_odd_cubic(Fast{}, 0.797884583f, 0.0356774069f, 0.107032225f, X));
+    return dual_half_one_plus_tanh(InRange{}, dual_odd_cubic(P{}, 0.797884583f, 0.0356774069f, 0.107032225f, X));
 }
 NFAD_DEV Gate<Wide> gate(Wide, GeluTanh, Seed X)
 {
@@ -284,13 +228,16 @@ NFAD_DEV Gate<Wide> gate(Wide, GeluTanh, Seed X)
 }
 
 // Swish (Table I, Table II): h = sigmoid(x)
-NFAD_DEV Gate<Fast> gate(Fast, Swish, Seed X) { return dual_sigmoid(Fast{}, InRange{}, X); }
+template <class P> NFAD_DEV Gate<P> gate(P, Swish, SeedOf<P> X) { return dual_sigmoid(P{}, InRange{}, X); }
 NFAD_DEV Gate<Wide> gate(Wide, Swish, Seed X) { return dual_sigmoid(Wide{}, X); }
 
 // Mish (Table I): h = tanh(softplus(x))
-template <class P> NFAD_DEV Gate<P> gate(P, Mish, Seed X) { return dual_tanh(dual_softplus(P{}, X)); }
+template <class P> NFAD_DEV Gate<P> gate(P, Mish, SeedOf<P> X) { return dual_tanh(dual_softplus(P{}, X)); }
+NFAD_DEV Gate<Wide> gate(Wide, Mish, Seed X) { return dual_tanh(dual_softplus(Wide{}, X)); }
 
-struct ActOut { float y, dydx; };
+template <class T> struct ActOutOf { T y, dydx; };
+using ActOut = ActOutOf<float>;
+using ActOut2 = ActOutOf<float2>;
 
 // x -> (f(x), f'(x)) in fp32, for any finite or non-finite x.  f = x h(x): the
 // last node of every chain is the product of the seed with the gate (v3 = v1 v2
@@ -307,40 +254,43 @@ template <class K> NFAD_DEV ActOut evaluate(K, Wide, float x)
     return {x > kSat ? x : y, dual_tangent(Y)};
 }
 
-template <class K> NFAD_DEV ActOut evaluate(K, Fast, float x)
+// Fast (one element) and Fast2 (two).  The gate and the tangent's product see the argument clamped to [kFastGateLo,
+// kFastGateHi], beyond which the gate is 0 or 1 and its slope 0 to every bit that a 16-bit result keeps.  The value's
+// product sees x itself, kept finite so that -inf gives -0; where the gate's range has no upper end, +inf becomes the
+// largest float, which rounds back to inf in either 16-bit type.
+template <class K, class P> NFAD_DEV ActOutOf<typename Lanes<P>::type> evaluate(K, P, typename Lanes<P>::type x)
 {
     using S = Saturation<K>;
     const float kMax = 3.40282347e+38f;
-    // The gate and the tangent's product see the argument clamped to [kFastGateLo, kFastGateHi], beyond which the gate is
-    // 0 or 1 and its slope 0 to every bit that a 16-bit result keeps.  The value's product sees x itself, kept finite so
-    // that -inf gives -0; where the gate's range has no upper end, +inf becomes the largest float, which rounds back to
-    // inf in either 16-bit type.
-    float xl, xg;
+    SeedOf<P> xl, xg;
     if (S::kFastGateHi >= kMax) {
-        xl = xg = hw::clamp_nan(x, S::kFastGateLo, kMax);
+        xl.x = xg.x = ln::clamp_nan(x, S::kFastGateLo, kMax);
     } else {
-        xl = hw::max_nan(x, -kMax);
-        xg = S::kFastGateLo > -kMax ? hw::clamp_nan(x, S::kFastGateLo, S::kFastGateHi) : hw::min_nan(xl, S::kFastGateHi);
+        xl.x = ln::max_nan(x, -kMax);
+        xg.x = S::kFastGateLo > -kMax ? ln::clamp_nan(x, S::kFastGateLo, S::kFastGateHi) : ln::min_nan(xl.x, S::kFastGateHi);
     }
-    Gate<Fast> H = gate(Fast{}, K{}, Seed{xg});
-    return {xl * H.v, fmaf(xg, H.t, H.v)};
+    Gate<P> Y = dual_mul(xl, xg, gate(P{}, K{}, xg));
+    return {Y.v, Y.t};
 }
 
 template <class K, class P> NFAD_DEV ActOut evaluate(float x) { return evaluate(K{}, P{}, x); }
 
 // x -> f(x) alone (a pass that will not be differentiated).  Same chain without the tangent parts; under the Fast
-// policy the gate's value may come from a cheaper form of the same accuracy class (value_gate), and only what the
+// policies the gate's value may come from a cheaper form of the same accuracy class (value_gate), and only what the
 // value needs is clamped: -inf becomes the most negative float so that 0 * x gives -0, +inf goes through as it is
 // (every gate is exactly 1 there) unless the gate's own range has an upper end.
-template <class K> NFAD_DEV float value_gate(K, float x) { return gate(Fast{}, K{}, Seed{x}).v; }
-NFAD_DEV float value_gate(GeluErf, float x) { return dual_half_one_plus_erf_scaled<4>(Fast{}, 0.707106769f, Seed{x}).v; }
+template <class K, class P> NFAD_DEV typename Lanes<P>::type value_gate(K, P, SeedOf<P> X) { return gate(P{}, K{}, X).v; }
+template <class P> NFAD_DEV typename Lanes<P>::type value_gate(GeluErf, P, SeedOf<P> X)
+{
+    return dual_half_one_plus_erf_scaled<4>(P{}, 0.707106769f, X).v;
+}
 template <class K> NFAD_DEV float evaluate_value(K, Wide, float x) { return evaluate(K{}, Wide{}, x).y; }
-template <class K> NFAD_DEV float evaluate_value(K, Fast, float x)
+template <class K, class P> NFAD_DEV typename Lanes<P>::type evaluate_value(K, P, typename Lanes<P>::type x)
 {
     using S = Saturation<K>;
-    const float xl = hw::max_nan(x, -3.40282347e+38f);
-    const float xg = S::kFastGateHi < 3.40282347e+38f ? hw::min_nan(xl, S::kFastGateHi) : xl;
-    return xl * value_gate(K{}, xg);
+    const auto xl = ln::max_nan(x, -3.40282347e+38f);
+    const auto xg = S::kFastGateHi < 3.40282347e+38f ? ln::min_nan(xl, S::kFastGateHi) : xl;
+    return ln::mul(xl, value_gate(K{}, P{}, SeedOf<P>{xg}));
 }
 
 // x -> h(x) alone (what a recomputation pass re-materialises).
@@ -349,10 +299,10 @@ template <class K> NFAD_DEV float evaluate_gate(K, Wide, float x)
     constexpr float kSat = Saturation<K>::kWide;
     return dual_value(gate(Wide{}, K{}, Seed{hw::clamp_nan(x, -kSat, kSat)}));
 }
-template <class K> NFAD_DEV float evaluate_gate(K, Fast, float x)
+template <class K, class P> NFAD_DEV typename Lanes<P>::type evaluate_gate(K, P, typename Lanes<P>::type x)
 {
     using S = Saturation<K>;
-    return gate(Fast{}, K{}, Seed{hw::clamp_nan(x, S::kFastGateLo, S::kFastGateHi)}).v;
+    return gate(P{}, K{}, SeedOf<P>{ln::clamp_nan(x, S::kFastGateLo, S::kFastGateHi)}).v;
 }
 template <class K, class P> NFAD_DEV float evaluate_gate(float x) { return evaluate_gate(K{}, P{}, x); }
 

@@ -89,6 +89,11 @@ NFAD_DEV double to_double(float x) { return double(x); }
 // double -> float, round to nearest even (subnormal results included)
 NFAD_DEV float to_float(double a) { return __double2float_rn(a); }
 
+// Packed fp32: two independent IEEE operations (round to nearest even) in one instruction.
+NFAD_DEV float2 fma2(float2 a, float2 b, float2 c) { return __ffma2_rn(a, b, c); }
+NFAD_DEV float2 mul2(float2 a, float2 b) { return __fmul2_rn(a, b); }
+NFAD_DEV float2 add2(float2 a, float2 b) { return __fadd2_rn(a, b); }
+
 NFAD_DEV int float_as_int(float a) { return __float_as_int(a); }
 NFAD_DEV float int_as_float(int a) { return __int_as_float(a); }
 

@@ -11,6 +11,11 @@ namespace nfad {
 // is the only tensor kept for back-propagation (Section II-C, approach 3).
 template <class P> struct IsFast { static constexpr bool value = false; };
 template <> struct IsFast<Fast> { static constexpr bool value = true; };
+// the chains that evaluate a polynomial (the cubic of GELU-tanh, the scaled erfc fit of GELU-erf): mostly fused
+// multiply-adds, which is what packed fp32 arithmetic halves
+template <class K> struct HasPolynomial { static constexpr bool value = false; };
+template <> struct HasPolynomial<GeluErf> { static constexpr bool value = true; };
+template <> struct HasPolynomial<GeluTanh> { static constexpr bool value = true; };
 
 template <class K, class P> struct ForwardTrainOp {
     static constexpr int kMinBlocks = 0;
@@ -26,19 +31,32 @@ template <class K, class P> struct ForwardTrainOp {
         out[0] = o.y;
         out[1] = o.dydx;
     }
+    // one element per call: with two outputs, pairs of registers per operand cost more (spills under the 48-register
+    // cap, or one resident CTA less) than the packed instructions save -- measured equal or 1-2 % slower
+    static constexpr bool kPairs = false;
 };
 
 // Forward, inference: x -> y.  Same chain; the tangent parts are dead code.
 template <class K, class P> struct ForwardInferOp {
-    static constexpr int kMinBlocks = 0;
-    // one input stream and one output: six packets per thread (16-bit storage) and eight (fp32 storage) measured 5-10 %
-    // faster than four
-    static constexpr int kUnroll = IsFast<P>::value ? 6 : 8;
+    // one input stream and one output.  16-bit storage, the two GELUs: two elements per call on packed fp32 arithmetic,
+    // eight packets per thread at four resident CTAs (64 registers: a pair of registers per operand needs the room);
+    // measured 0.90 / 0.94 of the copy peak (bf16; 0.86 / 0.92 fp16) against 0.85 / 0.89 (0.82 / 0.91) for one element
+    // per call in its best shape.  Swish and Mish (15 and 20 instructions per element, few of them multiply-adds) stay
+    // at one element per call, six packets and five CTAs: pairs measured within +-2 % there.  fp32 storage: eight
+    // packets, 5-10 % faster than four.
+    static constexpr bool kPairs = IsFast<P>::value && HasPolynomial<K>::value;
+    static constexpr int kMinBlocks = (IsFast<P>::value && !kPairs) ? 5 : 4;
+    static constexpr int kUnroll = (IsFast<P>::value && !kPairs) ? 6 : 8;
     static constexpr int kIn = 1, kOut = 1;
     static __device__ __forceinline__ constexpr bool keep(int) { return true; }
     static __device__ __forceinline__ void apply(const float (&in)[1], float (&out)[1])
     {
         out[0] = evaluate_value(K{}, P{}, in[0]);
+    }
+    // the same bits as apply on each element (the chain is one template for both widths)
+    static __device__ __forceinline__ void apply2(const float2 (&in)[1], float2 (&out)[1])
+    {
+        out[0] = evaluate_value(K{}, Fast2{}, in[0]);
     }
 };
 
@@ -62,6 +80,7 @@ struct BackwardOp {
     static constexpr int kUnroll = 0;
     static __device__ __forceinline__ constexpr bool keep(int) { return true; }
     static __device__ __forceinline__ void apply(const float (&in)[2], float (&out)[1]) { out[0] = __fmul_rn(in[0], in[1]); }
+    static constexpr bool kPairs = false;
 };
 
 // Conventional layout: x is saved, and backward re-derives f'(x) with the full
@@ -76,8 +95,9 @@ template <class K, class P> struct ConvBackwardOp {
     static __device__ __forceinline__ constexpr bool keep(int) { return true; }
     static __device__ __forceinline__ void apply(const float (&in)[2], float (&out)[1])
     {
-        out[0] = in[0] * evaluate<K, P>(in[1]).dydx;
+        out[0] = __fmul_rn(in[0], evaluate<K, P>(in[1]).dydx);
     }
+    static constexpr bool kPairs = false;       // two input streams already fill the registers: pairs measured 2-10 % slower
 };
 
 // Recomputation layout (Section II-C, approach 2): x is saved; backward first
@@ -85,13 +105,19 @@ template <class K, class P> struct ConvBackwardOp {
 // per-operator backward rules need (the gate h = v1 of the Swish example), then
 // walks those rules: x' = g v1 + g v2 v1' with v2 = x (Eq. 2).
 template <class K, class P> struct RecomputePhase1Op {
-    static constexpr int kMinBlocks = 0;
-    static constexpr int kUnroll = IsFast<P>::value ? 6 : 8;      // the same shape as the value-only forward
+    // the same widths and tile shapes as the value-only forward
+    static constexpr bool kPairs = ForwardInferOp<K, P>::kPairs;
+    static constexpr int kMinBlocks = ForwardInferOp<K, P>::kMinBlocks;
+    static constexpr int kUnroll = ForwardInferOp<K, P>::kUnroll;
     static constexpr int kIn = 1, kOut = 1;
     static __device__ __forceinline__ constexpr bool keep(int) { return true; }
     static __device__ __forceinline__ void apply(const float (&in)[1], float (&out)[1])
     {
         out[0] = evaluate_gate<K, P>(in[0]);
+    }
+    static __device__ __forceinline__ void apply2(const float2 (&in)[1], float2 (&out)[1])
+    {
+        out[0] = evaluate_gate(K{}, Fast2{}, in[0]);
     }
 };
 
@@ -138,6 +164,7 @@ template <class K, class P> struct RecomputePhase2Op {
         float hs = GateSlope<K>::of(x, h);
         out[0] = fmaf(g * x, hs, g * h);
     }
+    static constexpr bool kPairs = false;
 };
 
 // Traffic probe: moves bytes through the same streaming engine with no arithmetic to speak
@@ -154,6 +181,7 @@ template <int NIN, int NOUT> struct ProbeOp {
         out[0] = v;
         if (NOUT > 1) out[1] = __uint_as_float(~__float_as_uint(v));
     }
+    static constexpr bool kPairs = false;
 };
 
 }  // namespace nfad

@@ -37,7 +37,9 @@ template <int NIN, int NOUT> struct StreamArgs {
 //   static constexpr int kIn, kOut;  static constexpr bool keep(int out_slot);
 //   static __device__ void apply(const float (&in)[kIn], float (&out)[kOut]);
 //   static constexpr int kMinBlocks: resident CTAs per SM to leave room for (0: the storage type's default);
-//   static constexpr int kUnroll: packets per thread and tile (0: the default, 4).
+//   static constexpr int kUnroll: packets per thread and tile (0: the default, 4);
+//   static constexpr bool kPairs; if set, apply2(const float2 (&in)[kIn], float2 (&out)[kOut]) does two elements at once
+//   with the same results as apply on each (packed fp32 arithmetic: half the issue slots for multiplies and adds).
 template <class S, class Op>
 __device__ __forceinline__ void scalar_element(const StreamArgs<Op::kIn, Op::kOut>& a, size_t i)
 {
@@ -59,14 +61,26 @@ __device__ __forceinline__ void packet_compute_store(const StreamArgs<Op::kIn, O
     float vout[Op::kOut][V];
 #pragma unroll
     for (int k = 0; k < Op::kIn; ++k) S::unpack(raw[k], vin[k]);
+    if constexpr (Op::kPairs) {                 // two elements per call on packed fp32 arithmetic
 #pragma unroll
-    for (int e = 0; e < V; ++e) {
-        float in[Op::kIn], out[Op::kOut];
+        for (int e = 0; e < V; e += 2) {
+            float2 in[Op::kIn], out[Op::kOut];
 #pragma unroll
-        for (int k = 0; k < Op::kIn; ++k) in[k] = vin[k][e];
-        Op::apply(in, out);
+            for (int k = 0; k < Op::kIn; ++k) in[k] = make_float2(vin[k][e], vin[k][e + 1]);
+            Op::apply2(in, out);
 #pragma unroll
-        for (int k = 0; k < Op::kOut; ++k) vout[k][e] = out[k];
+            for (int k = 0; k < Op::kOut; ++k) { vout[k][e] = out[k].x; vout[k][e + 1] = out[k].y; }
+        }
+    } else {
+#pragma unroll
+        for (int e = 0; e < V; ++e) {
+            float in[Op::kIn], out[Op::kOut];
+#pragma unroll
+            for (int k = 0; k < Op::kIn; ++k) in[k] = vin[k][e];
+            Op::apply(in, out);
+#pragma unroll
+            for (int k = 0; k < Op::kOut; ++k) vout[k][e] = out[k];
+        }
     }
     const size_t byte_off = a.head * sizeof(typename S::elem);
 #pragma unroll

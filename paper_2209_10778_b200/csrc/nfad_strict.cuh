@@ -41,6 +41,7 @@ template <class K> struct ForwardStrictOp {
     static constexpr int kMinBlocks = 0;
     static constexpr int kUnroll = 4;
     static constexpr int kIn = 1, kOut = 2;
+    static constexpr bool kPairs = false;
     static __device__ __forceinline__ constexpr bool keep(int k) { return k == 0; }
     static __device__ __forceinline__ void apply(const float (&in)[1], float (&out)[2])
     {

@@ -68,6 +68,28 @@ def test_unaligned_and_misaligned_pointers_give_identical_bits(dtype):
         assert (db[:od] == 7.0).all() and (db[od + n:] == 7.0).all()
 
 
+@pytest.mark.parametrize("kind", KINDS)
+@pytest.mark.parametrize("dtype", ["bf16", "f16"])
+def test_value_only_forward_is_the_same_on_every_path(kind, dtype):
+    """The value-only forward of 16-bit storage runs two elements per call on packed fp32 arithmetic where the
+    pointers allow whole packets, and one element per call otherwise (ragged ends, mutually misaligned pointers):
+    over every finite value of the type (and the non-finite ones) the two must agree bit for bit."""
+    td = W.TORCH_DTYPES[dtype]
+    fin = W.all_finite_16bit(dtype)
+    special = torch.tensor([float("inf"), float("-inf"), float("nan")], dtype=td)
+    x0 = torch.cat([fin, special, fin.flip(0)]).to(DEV)          # odd length: a ragged tail on the packet path
+    n = x0.numel()
+    y0 = torch.empty_like(x0)
+    nfad.nfad_act_forward_infer(kind, x0, y0)                    # aligned: packets
+    xb = torch.zeros(n + 16, dtype=td, device=DEV)
+    yb = torch.full((n + 16,), 7.0, dtype=td, device=DEV)
+    xb[1:1 + n] = x0
+    nfad.nfad_act_forward_infer(kind, xb[1:1 + n], yb[2:2 + n])  # offsets differ modulo a packet: element by element
+    torch.cuda.synchronize()
+    assert ulp.same_bits_or_both_nan(W.raw_numpy(yb[2:2 + n]), W.raw_numpy(y0), dtype).all()
+    assert (yb[:2] == 7.0).all() and (yb[2 + n:] == 7.0).all()
+
+
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 def test_in_place(dtype):
     n = 50001
