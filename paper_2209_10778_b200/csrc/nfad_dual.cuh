@@ -222,9 +222,11 @@ template <class P> NFAD_DEV Gate<P> gate(P, GeluTanh, SeedOf<P> X)
 {
     return dual_half_one_plus_tanh(InRange{}, dual_odd_cubic(P{}, 0.797884583f, 0.0356774069f, 0.107032225f, X));
 }
+// Wide: (1 + tanh u)/2 = sigmoid(2u), with the 2 folded into the cubic's constants (a scale by a constant is unary,
+// Section III-A; doubling is exact)
 NFAD_DEV Gate<Wide> gate(Wide, GeluTanh, Seed X)
 {
-    return dual_half_one_plus_tanh(InRange{}, dual_odd_cubic(Wide{}, 0.7978845608028654, 0.035677408136300125, 0.10703222440890037, X));
+    return dual_sigmoid(InRange{}, dual_odd_cubic(Wide{}, 2.0 * 0.7978845608028654, 2.0 * 0.035677408136300125, 2.0 * 0.10703222440890037, X));
 }
 
 // Swish (Table I, Table II): h = sigmoid(x)

@@ -72,6 +72,27 @@ template <int kDegree> NFAD_DEV double exp_bounded(double a)
 }
 NFAD_DEV double exp_neg(double a) { return exp_bounded<11>(a); }
 
+// kappa e^(-g s) for s >= 0 with g s <= 700, to 2^-29: the degree-6 form of exp_bounded with both constants folded in,
+// so that neither costs an operation.  -g s = n ln2 + r with r = -g r', r' = s + n ln2/g: the polynomial runs in r'
+// with its coefficients multiplied by kappa (-g)^i (g and kappa are compile-time constants at every call).
+NFAD_DEV double exp_neg_scaled(double s, double g, double kappa)
+{
+    const double kMagic = 6755399441055744.0;
+    double t = fma(s, -g * 1.4426950408889634, kMagic);
+    double n = t - kMagic;
+    int ni = hw::double_lo(t);
+    double rp = fma(n, 0.6931471805599453 / g, s);
+    const double m = -g;
+    double p = kappa * 0.0013836846134577057 * (m * m * m * m * m * m);
+    p = fma(p, rp, kappa * 0.008374815798301793 * (m * m * m * m * m));
+    p = fma(p, rp, kappa * 0.04166822556692284 * (m * m * m * m));
+    p = fma(p, rp, kappa * 0.16666420169946367 * (m * m * m));
+    p = fma(p, rp, kappa * 0.4999999207982802 * (m * m));
+    p = fma(p, rp, kappa * 1.0000000363231765 * m);
+    p = fma(p, rp, kappa * 1.0000000005541663);
+    return hw::double_from(hw::double_hi(p) + (ni << 20), hw::double_lo(p));
+}
+
 // erfc(z)/2 = exp(-z^2) W(z) for z >= 0.  W(z) (z + k) is a smooth function of q = (z - k)/(z + k) in [-1, 1), fitted
 // by one polynomial on z in [0, 15], k = 3/sqrt(2).  Returns W(z); the caller owns the exponential, so that value and
 // slope share it.
@@ -95,10 +116,11 @@ NFAD_DEV double half_erfcx(double z)
     for (int i = 21; i >= 0; --i) p = fma(p, q, c[i]);
     return p * r;
 }
-NFAD_DEV double half_erfcx_mix(double z_plus_k)
+// The argument is kappa (z + k) and the result W(z)/kappa, for any constant kappa > 0 the caller wants folded in.
+NFAD_DEV double half_erfcx_mix(double z_plus_k_scaled, double kappa)
 {
-    double r = rcp<1>(z_plus_k);
-    float q = hw::to_float(fma(-2.0 * 2.1213202476501465, r, 1.0));
+    double r = rcp<1>(z_plus_k_scaled);                                          // 1/(kappa (z + k))
+    float q = hw::to_float(fma(-2.0 * 2.1213202476501465 * kappa, r, 1.0));      // (z - k)/(z + k)
     float p = 4.23795245e-05f;
     p = fmaf(p, q, 9.49347959e-05f);
     p = fmaf(p, q, -0.0001815203f);
@@ -186,8 +208,9 @@ NFAD_DEV double clamp700(double v) { return v != v ? v : fmin(fmax(v, -700.0), 7
 NFAD_DEV Gate<Wide> dual_sigmoid(Wide, const Seed& a) { return logistic_wide<false>(hw::to_double(a.x), 1.0); }
 NFAD_DEV Gate<Wide> dual_sigmoid(const Dual<Wide>& a) { return logistic_wide<true>(clamp700(a.v), a.t); }
 
+NFAD_DEV Gate<Wide> dual_sigmoid(InRange, const Dual<Wide>& a) { return logistic_wide<false>(a.v, a.t); }
+
 // (1 + tanh u)/2 = L(2u), slope 2 L'(2u)
-NFAD_DEV Gate<Wide> dual_half_one_plus_tanh(InRange, const Dual<Wide>& u) { return logistic_wide<false>(u.v + u.v, u.t + u.t); }
 NFAD_DEV Gate<Wide> dual_half_one_plus_tanh(const Dual<Wide>& u) { return logistic_wide<true>(clamp700(u.v + u.v), u.t + u.t); }
 
 // (1 + erf z)/2 = erfc(-z)/2: with E = exp(-z^2) and W = erfcx(|z|)/2 it is E W for z < 0 and 1 - E W for z >= 0;
@@ -203,10 +226,11 @@ NFAD_DEV Gate<Wide> dual_half_one_plus_erf(const Dual<Wide>& z)
 // Section III-A), so that -c^2 x^2 and c |x| + k each are one operation.  |c x| <= 15.
 NFAD_DEV Gate<Wide> dual_half_one_plus_erf_scaled(Wide, double c, const Seed& a)
 {
+    const double kappa = 0.5641895835477563 * c;             // the slope is kappa E: E is formed times kappa, W over kappa
     double x = hw::to_double(a.x);
-    double E = wide::exp_bounded<6>((x * x) * -(c * c));
-    double v = E * wide::half_erfcx_mix(fma(fabs(x), c, 2.1213202476501465));
-    return {a.x < 0.0f ? v : 1.0 - v, E * (0.5641895835477563 * c)};
+    double Ek = wide::exp_neg_scaled(x * x, c * c, kappa);
+    double v = Ek * wide::half_erfcx_mix(fma(fabs(x), c * kappa, 2.1213202476501465 * kappa), kappa);
+    return {a.x < 0.0f ? v : 1.0 - v, Ek};
 }
 
 // ----------------------------------------------------------------- softplus, and tanh of a softplus
