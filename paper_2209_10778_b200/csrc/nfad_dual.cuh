@@ -218,12 +218,12 @@ NFAD_DEV Gate<Wide> gate(Wide, GeluErf, Seed X) { return dual_half_one_plus_erf_
 
 // GELU, tanh form (Table I): h = (1 + tanh(sqrt(2/pi) (x + 0.044715 x^3)))/2
 //   u = c x + (c a) x^3 with c = sqrt(2/pi), a = 0.044715 (the double nearest to it); the last constant is 3 c a
+//   (1 + tanh u)/2 = sigmoid(2u), and the 2 goes into the cubic's constants (a scale by a constant is unary, Section
+//   III-A; doubling is exact, so the value is bit for bit that of (1 + tanh u)/2 formed from u)
 template <class P> NFAD_DEV Gate<P> gate(P, GeluTanh, SeedOf<P> X)
 {
-    return dual_half_one_plus_tanh(InRange{}, dual_odd_cubic(P{}, 0.797884583f, 0.0356774069f, 0.107032225f, X));
+    return dual_sigmoid(InRange{}, dual_odd_cubic(P{}, 2.0f * 0.797884583f, 2.0f * 0.0356774069f, 2.0f * 0.107032225f, X));
 }
-// Wide: (1 + tanh u)/2 = sigmoid(2u), with the 2 folded into the cubic's constants (a scale by a constant is unary,
-// Section III-A; doubling is exact)
 NFAD_DEV Gate<Wide> gate(Wide, GeluTanh, Seed X)
 {
     return dual_sigmoid(InRange{}, dual_odd_cubic(Wide{}, 2.0 * 0.7978845608028654, 2.0 * 0.035677408136300125, 2.0 * 0.10703222440890037, X));

@@ -90,13 +90,13 @@ template <class P> NFAD_DEV Gate<P> dual_sigmoid(P, InRange, const SeedOf<P>& a)
     auto L = ln::mul(r, kTwoPowMinus64);
     return {L, ln::mul(L, ln::mul(E, r))};
 }
-// H = (1 + tanh u)/2 = L(2u),  dH/dx = 2 L'(2u) u'   [= (1 - tanh^2 u) u'/2]
-template <class P> NFAD_DEV Gate<P> dual_half_one_plus_tanh(InRange, const Dual<P>& u)
+// sigmoid of a dual w (the caller keeps w.v >= -133): the slope is L (E r) w'.  (1 + tanh u)/2 is this with w = 2u.
+template <class P> NFAD_DEV Gate<P> dual_sigmoid(InRange, const Dual<P>& w)
 {
-    auto E = ln::ex2_ftz(ln::fma(u.v, -2.88539004f, -64.0f));
+    auto E = ln::ex2_ftz(ln::fma(w.v, -1.44269502f, -64.0f));
     auto r = ln::rcp(ln::add(E, kTwoPowMinus64));
     auto L = ln::mul(r, kTwoPowMinus64);
-    return {L, ln::mul(ln::mul(L, ln::mul(E, r)), ln::mul(u.t, 2.0f))};
+    return {L, ln::mul(ln::mul(L, ln::mul(E, r)), w.t)};
 }
 
 // 2^-64 W(z) from r = 1/(z + k): the fit described at half_erfcx_fast_scaled (nfad_numerics.cuh), per lane
@@ -144,15 +144,15 @@ template <class P> NFAD_DEV SoftplusDual<P> dual_softplus(P, const SeedOf<P>& a)
     return {ln::mul(ln::ex2_ftz(ln::fma(a.x, 1.44269502f, 64.0f)), kTwoPowMinus64)};
 }
 // tanh(log1p(w)) = ((1+w)^2 - 1)/((1+w)^2 + 1) = n/(n + 2), n = w (w + 2): one form for both signs, every term
-// positive.  T' = (dn/dx) 2/(n + 2)^2 = 4 w (w + 1)/(n + 2)^2.  Needs w <= 2^29 (x <= 20), so that the factors of
-// the slope stay inside fp32's range.
+// positive.  T' = (dn/dx) 2/(n + 2)^2 = 4 w (w + 1)/(n + 2)^2.  Formed with the halves h = (w + 2)/2, m = n/2 = w h and
+// r = 2/(n + 2) = 1/(w h + 1), so that no factor 2 or 4 costs an operation:  T = m r,  T' = (w r) (w r + r).
+// Needs w <= 2^29 (x <= 20), so that the factors stay inside fp32's range.
 template <class P> NFAD_DEV Gate<P> dual_tanh_of_softplus(const SoftplusDual<P>& p)
 {
     auto w = p.w;
-    auto w2 = ln::add(w, 2.0f);
-    auto n = ln::mul(w, w2);
-    auto rd = ln::rcp(ln::fma(w, w2, 2.0f));
-    return {ln::mul(n, rd), ln::mul(ln::mul(ln::mul(w, rd), 4.0f), ln::mul(ln::add(w, 1.0f), rd))};
+    auto h = ln::fma(w, 0.5f, 1.0f);
+    auto r = ln::rcp(ln::fma(w, h, 1.0f));
+    return {ln::mul(ln::mul(w, h), r), ln::mul(ln::mul(w, r), ln::fma(w, r, r))};
 }
 NFAD_DEV Gate<Fast> dual_tanh(const SoftplusDual<Fast>& p) { return dual_tanh_of_softplus<Fast>(p); }
 NFAD_DEV Gate<Fast2> dual_tanh(const SoftplusDual<Fast2>& p) { return dual_tanh_of_softplus<Fast2>(p); }
