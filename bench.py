@@ -199,6 +199,16 @@ class _Timer:
                 "launches_per_burst": per_burst * launches_per_replay, "bursts": repeats, "wall": (t0, t1)}
 
 
+MAX_GRAPH_STEPS = 256          # steps captured into one graph (4 launches each for the headline workload)
+GRAPH_LAUNCHES = 48            # launches per graph when one kernel is timed alone
+
+
+def _graph_cycles(n_sets: int) -> int:
+    """How often a per-kernel graph walks the buffer sets: about GRAPH_LAUNCHES launches per replay, so that the gap
+    between two replays (the one kernel boundary that is not a programmatic dependent launch) stays below 1 % of it."""
+    return max(1, GRAPH_LAUNCHES // n_sets)
+
+
 def _launcher(nfad, kind, op, scratch=None):
     """set -> one launch of `op` on that buffer set."""
     if op == "forward":
@@ -290,21 +300,25 @@ def run_ours(args, w):
             nfad.nfad_act_forward(kind, a["x"], a["y"], a["d"])
             nfad.nfad_act_backward(kind, b["g"], b["d"], b["gin"])
 
-    # after `period` steps every launch sees the buffers of `period` steps ago
+    # after `period` steps every launch sees the buffers of `period` steps ago.  A region is one graph of all K steps
+    # (chunks of at most MAX_GRAPH_STEPS, whole periods, for a very large K): every kernel boundary inside it is a
+    # programmatic dependent launch, as it is in a training step that launches its kernels back to back.
     period = n_sets // math.gcd(n_sets, len(kinds))
-    full, rem = divmod(args.steps, period)
-    replay_period = timer.graph(lambda: [step(i) for i in range(period)])
-    replay_rem = timer.graph(lambda: [step(i) for i in range(rem)]) if rem else None
+    chunk = args.steps if args.steps <= MAX_GRAPH_STEPS else period * max(1, MAX_GRAPH_STEPS // period)
+    full, rem = divmod(args.steps, chunk)
+    replay_chunk = timer.graph(lambda: [step(i) for i in range(chunk)])
+    replay_rem = timer.graph(lambda: [step(full * chunk + i) for i in range(rem)]) if rem else None
 
     def region():
         for _ in range(full):
-            replay_period()
+            replay_chunk()
         if replay_rem:
             replay_rem()
 
     warm = max(3, args.warmup)
+    replay_warm = timer.graph(lambda: [step(i) for i in range(period)])
     for _ in range(-(-warm // period)):
-        replay_period()
+        replay_warm()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     region()
@@ -330,11 +344,12 @@ def run_ours(args, w):
 
     # ------------------------------------------------------------------ the step's kernels, one by one (after the regions)
     step_kernels = {}
+    cycles = _graph_cycles(n_sets)
     for kind in kinds:
         for op in ("forward", "backward"):
             fn = _launcher(nfad, kind, op)
-            replay = timer.graph(lambda: [fn(s) for s in sets])
-            r = timer.bursts(replay, n_sets)
+            replay = timer.graph(lambda: [fn(s) for _ in range(cycles) for s in sets])
+            r = timer.bursts(replay, cycles * n_sets)
             c = clocks_between(*r["wall"], "")
             step_kernels[f"{kind}_{op}"] = (r, c["sm_mhz"] if c and c["samples"] else None)
 
@@ -398,8 +413,9 @@ def run_ours(args, w):
                 for op, table in (("forward", per_kernel), ("infer", per_kernel), ("backward", per_kernel),
                                   ("conv_backward", comparators), ("recompute_backward", comparators)):
                     fn = _launcher(nfad, kind, op, scratch)
-                    replay = timer.graph(lambda: [fn(s) for s in tsets])
-                    r = timer.bursts(replay, len(tsets), min_burst_ms=30.0)
+                    cyc = _graph_cycles(len(tsets))
+                    replay = timer.graph(lambda: [fn(s) for _ in range(cyc) for s in tsets])
+                    r = timer.bursts(replay, cyc * len(tsets), min_burst_ms=30.0)
                     c = clocks_between(*r["wall"], "")
                     table[f"{kind}_{dtype}_{op}"] = _kernel_entry(r, op, esd, n_big, peak, c["sm_mhz"] if c and c["samples"] else None)
                 del scratch
@@ -429,8 +445,9 @@ def run_ours(args, w):
         "frac_of_nominal_8000": achieved / 8000.0,
         "algorithmic_bytes_per_launch": algo_bytes, "avg_launch_ms": dom_r["ms"],
         "sm_mhz": dom_mhz, "kcycles_per_launch": round(dom_r["ms"] * dom_mhz, 2) if dom_mhz else None,
-        "timing": f"after the headline regions: the kernel replayed back to back from a graph over the {n_sets} buffer sets, "
-                  f"median of {dom_r['bursts']} bursts of {dom_r['launches_per_burst']} launches (>= 20 ms each)",
+        "timing": f"after the headline regions: the kernel replayed back to back from a graph of {cycles * n_sets} launches "
+                  f"walking the {n_sets} buffer sets, median of {dom_r['bursts']} bursts of {dom_r['launches_per_burst']} "
+                  "launches (>= 20 ms each)",
         "traffic": (tpe * n) if tpe else None,
         "traffic_source": "ncu dram bytes per element at n = 2^26 (profiles/) x the elements of this launch",
         "step": {"algorithmic_bytes": step_bytes, "achieved": step_gbs, "frac": step_gbs / peak,
@@ -466,8 +483,9 @@ def run_ours(args, w):
         "roofline": roofline, "cpu_baseline": cpu_baseline, "e2e": e2e,
         "gpu_launches": 2 * len(kinds) * args.steps * R,
         "gpu_launches_per_region": 2 * len(kinds) * args.steps,
-        "launch": (f"CUDA graph of one buffer-rotation period ({period} steps, {2 * len(kinds) * period} kernels, programmatic "
-                   "dependent launch between them)" if not args.no_graph else "every kernel launched from the host"),
+        "launch": (f"one CUDA graph per {chunk} steps ({2 * len(kinds) * chunk} kernels, programmatic dependent launch between "
+                   f"them; the buffers rotate with a period of {period} steps)" if not args.no_graph
+                   else "every kernel launched from the host"),
         "per_kernel": per_kernel, "comparators": comparators, "stack": stack, "bert_base_ffn": bert,
         "per_kernel_note": (f"n = {n_big} elements per tensor, x ~ N(0,1); median of 10 bursts >= 30 ms of graph-replayed "
                             "back-to-back launches; frac = algorithmic GB/s over the peak above; kcycles = ms x the median SM MHz "
@@ -595,8 +613,9 @@ def _small_workload_section(torch, nfad, W, timer, dev, peak, w, clocks_between)
             nfad.nfad_act_backward(kind, b["g"], b["d"], b["gin"])
 
     period = n_sets // math.gcd(n_sets, len(kinds))
-    replay = timer.graph(lambda: [step(i) for i in range(period)])
-    r = timer.bursts(replay, period)               # ms per step
+    g_steps = period * max(1, (2 * GRAPH_LAUNCHES) // (2 * len(kinds) * period))
+    replay = timer.graph(lambda: [step(i) for i in range(g_steps)])
+    r = timer.bursts(replay, g_steps)              # ms per step
     step_bytes = 2 * len(kinds) * 3 * es * n
     out = {"shape": list(w.shapes[0]), "elements": n, "dtype": w.dtype, "kinds": kinds, "ms_per_step": r["ms"],
            "elements_per_s": n * len(kinds) / (r["ms"] / 1e3), "step_GBps": step_bytes / (r["ms"] / 1e3) / 1e9,
@@ -604,7 +623,8 @@ def _small_workload_section(torch, nfad, W, timer, dev, peak, w, clocks_between)
     for kind in kinds:
         for op in ("forward", "backward"):
             fn = _launcher(nfad, kind, op)
-            rk = timer.bursts(timer.graph(lambda: [fn(s) for s in sets]), n_sets)
+            cyc = _graph_cycles(n_sets)
+            rk = timer.bursts(timer.graph(lambda: [fn(s) for _ in range(cyc) for s in sets]), cyc * n_sets)
             c = clocks_between(*rk["wall"], "")
             out["kernels"][f"{kind}_{op}"] = _kernel_entry(rk, op, es, n, peak, c["sm_mhz"] if c and c["samples"] else None)
     del sets
