@@ -17,12 +17,22 @@ template <class K> struct HasPolynomial { static constexpr bool value = false; }
 template <> struct HasPolynomial<GeluErf> { static constexpr bool value = true; };
 template <> struct HasPolynomial<GeluTanh> { static constexpr bool value = true; };
 
+template <class K> struct IsErf { static constexpr bool value = false; };
+template <> struct IsErf<GeluErf> { static constexpr bool value = true; };
+
 template <class K, class P> struct ForwardTrainOp {
     static constexpr int kMinBlocks = 0;
+    // 16-bit storage, GELU-erf (the longest chain: 25 instructions per element, 16 of them multiply-adds): two elements
+    // per call on packed fp32 arithmetic (18 instructions per element).  With four packets per thread the pairs fit the
+    // 48-register cap without spills (five packets spill 48-56 bytes), and under a sustained load, where the clock sags
+    // and this kernel is short of issue slots, that is worth 2 points for bf16 (0.925 -> 0.945 of the copy peak in the
+    // benchmark's own timing) and 4 for fp16.  The other three chains are not short of issue slots: pairs measured
+    // equal or 1-5 % slower for them (spills, or one resident CTA less), so they stay at one element per call.
+    static constexpr bool kPairs = IsFast<P>::value && IsErf<K>::value;
     // packets per thread and tile, measured at 100.7M elements: 16-bit storage 5 (1-4 % faster than 4; 3 and 6 are slower
-    // under the 48-register cap), fp32 storage 7 (0.76 / 0.82 / 0.95 / 0.87 of the copy peak against 0.72 / 0.82 / 0.88 /
-    // 0.84 with 4; 8 and 10 fall off again)
-    static constexpr int kUnroll = IsFast<P>::value ? 5 : 7;
+    // under the 48-register cap), 4 with pairs; fp32 storage 7 (0.76 / 0.82 / 0.95 / 0.87 of the copy peak against 0.72 /
+    // 0.82 / 0.88 / 0.84 with 4; 8 and 10 fall off again)
+    static constexpr int kUnroll = IsFast<P>::value ? (kPairs ? 4 : 5) : 7;
     static constexpr int kIn = 1, kOut = 2;
     static __device__ __forceinline__ constexpr bool keep(int k) { return k == 0; }   // y is consumed next; f' much later
     static __device__ __forceinline__ void apply(const float (&in)[1], float (&out)[2])
@@ -31,9 +41,13 @@ template <class K, class P> struct ForwardTrainOp {
         out[0] = o.y;
         out[1] = o.dydx;
     }
-    // one element per call: with two outputs, pairs of registers per operand cost more (spills under the 48-register
-    // cap, or one resident CTA less) than the packed instructions save -- measured equal or 1-2 % slower
-    static constexpr bool kPairs = false;
+    // the same bits as apply on each element (the chain is one template for both widths)
+    static __device__ __forceinline__ void apply2(const float2 (&in)[1], float2 (&out)[2])
+    {
+        ActOut2 o = evaluate(K{}, Fast2{}, in[0]);
+        out[0] = o.y;
+        out[1] = o.dydx;
+    }
 };
 
 // Forward, inference: x -> y.  Same chain; the tangent parts are dead code.

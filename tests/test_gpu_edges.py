@@ -47,11 +47,11 @@ def test_sizes_and_guard_bands(dtype):
             parity.check_backward(dtype, W.raw_numpy(g), W.raw_numpy(d), W.raw_numpy(gin))
 
 
+@pytest.mark.parametrize("kind", ["mish", "gelu_erf"])      # one element per call; two per call in whole packets (16-bit)
 @pytest.mark.parametrize("dtype", ["f32", "bf16", "f16"])
-def test_unaligned_and_misaligned_pointers_give_identical_bits(dtype):
+def test_unaligned_and_misaligned_pointers_give_identical_bits(dtype, kind):
     td = W.TORCH_DTYPES[dtype]
     n = 20011
-    kind = "mish"
     x0 = W.draw("mix", n, dtype, 11, DEV)
     y0, d0 = parity.gpu_forward(kind, x0)
     per16 = 16 // x0.element_size()
@@ -88,6 +88,26 @@ def test_value_only_forward_is_the_same_on_every_path(kind, dtype):
     torch.cuda.synchronize()
     assert ulp.same_bits_or_both_nan(W.raw_numpy(yb[2:2 + n]), W.raw_numpy(y0), dtype).all()
     assert (yb[:2] == 7.0).all() and (yb[2 + n:] == 7.0).all()
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f16"])
+def test_training_forward_is_the_same_on_every_path(dtype):
+    """GELU-erf's training forward runs two elements per call in whole packets and one per call elsewhere: over
+    every value of the type both outputs must agree bit for bit."""
+    td = W.TORCH_DTYPES[dtype]
+    fin = W.all_finite_16bit(dtype)
+    special = torch.tensor([float("inf"), float("-inf"), float("nan")], dtype=td)
+    x0 = torch.cat([fin, special, fin.flip(0)]).to(DEV)
+    n = x0.numel()
+    y0, d0 = parity.gpu_forward("gelu_erf", x0)                   # aligned: packets
+    xb = torch.zeros(n + 16, dtype=td, device=DEV)
+    yb = torch.full((n + 16,), 7.0, dtype=td, device=DEV)
+    db = torch.full((n + 16,), 7.0, dtype=td, device=DEV)
+    xb[1:1 + n] = x0
+    nfad.nfad_act_forward("gelu_erf", xb[1:1 + n], yb[2:2 + n], db[3:3 + n])   # no common packet grid: element by element
+    torch.cuda.synchronize()
+    assert ulp.same_bits_or_both_nan(W.raw_numpy(yb[2:2 + n]), W.raw_numpy(y0), dtype).all()
+    assert ulp.same_bits_or_both_nan(W.raw_numpy(db[3:3 + n]), W.raw_numpy(d0), dtype).all()
 
 
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
