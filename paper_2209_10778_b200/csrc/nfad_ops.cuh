@@ -102,16 +102,21 @@ struct BackwardOp {
 template <class K, class P> struct ConvBackwardOp {
     // two input streams: their packets alone are 24-40 registers, so room for 64 (four resident CTAs) or the chain's
     // temporaries spill.  Packets per thread, measured at 100.7M elements: 16-bit storage 5 (0.90-1.02 of the copy peak
-    // against 0.80-0.89 with 4), fp32 storage 3 (0.72-0.91 against 0.70-0.87)
+    // against 0.80-0.89 with 4), fp32 storage 3 (0.72-0.91 against 0.70-0.87).  GELU-erf, 16-bit storage: two elements
+    // per call as in the training forward, three packets per thread (more spill): 0.87 -> 0.88 bf16, 0.86 -> 0.88 fp16.
+    static constexpr bool kPairs = IsFast<P>::value && IsErf<K>::value;
     static constexpr int kMinBlocks = 4;
-    static constexpr int kUnroll = IsFast<P>::value ? 5 : 3;
+    static constexpr int kUnroll = IsFast<P>::value ? (kPairs ? 3 : 5) : 3;
     static constexpr int kIn = 2, kOut = 1;
     static __device__ __forceinline__ constexpr bool keep(int) { return true; }
     static __device__ __forceinline__ void apply(const float (&in)[2], float (&out)[1])
     {
         out[0] = __fmul_rn(in[0], evaluate<K, P>(in[1]).dydx);
     }
-    static constexpr bool kPairs = false;       // two input streams already fill the registers: pairs measured 2-10 % slower
+    static __device__ __forceinline__ void apply2(const float2 (&in)[2], float2 (&out)[1])
+    {
+        out[0] = hw::mul2(in[0], evaluate(K{}, Fast2{}, in[1]).dydx);
+    }
 };
 
 // Recomputation layout (Section II-C, approach 2): x is saved; backward first
