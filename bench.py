@@ -52,8 +52,8 @@ DTYPES = ("f32", "bf16", "f16")
 # elements) measured by ncu at n = 2^26, where every tensor exceeds L2; summarised under profiles/.
 # Traffic grows in proportion to n, so a launch's traffic is this figure times its elements.
 NCU_TRAFFIC_BYTES_PER_ELEMENT = {
-    "gelu_erf_bf16_forward": 5.124, "gelu_tanh_bf16_forward": 5.142, "swish_bf16_forward": 5.131,
-    "mish_bf16_forward": 5.152, "bf16_backward": 5.190,
+    "gelu_erf_bf16_forward": 5.138, "gelu_tanh_bf16_forward": 5.135, "swish_bf16_forward": 5.141,
+    "mish_bf16_forward": 5.159, "bf16_backward": 5.184,
 }
 # tensors read, written per element
 OP_TENSORS = {"forward": (1, 2), "infer": (1, 1), "backward": (2, 1), "conv_backward": (2, 1),

@@ -5,9 +5,9 @@
 // element, more than half of them fp32 multiplies, adds and fused multiply-adds.  sm_100 has packed forms of those
 // three (fma.rn.f32x2 and friends: two independent IEEE operations, one issue slot), so the same chain on a pair of
 // elements needs half the issue slots for that part.  What has no packed form (the exponential and reciprocal units,
-// min / max, selects, |x|) is issued once per lane, and a pair of registers per operand costs registers: the
-// value-only forward gains 3 to 5 % from pairs, the two-output forward and the backward kernels do not, so each
-// kernel picks its width (nfad_ops.cuh).
+// min / max, selects, |x|) is issued once per lane, and a pair of registers per operand costs registers: pairs pay
+// where a chain is long enough to be short of issue slots and a tile shape holds them without spilling (the GELU-erf
+// kernels, the value-only GELU-tanh), and cost a few per cent elsewhere, so each kernel picks its width (nfad_ops.cuh).
 //
 // Every function below is a template over the policy and calls only the `ln::` operations, each of which is the same
 // IEEE operation per lane in both widths (explicit fma / mul / add: nothing is left to contraction).  A lane of a pair
