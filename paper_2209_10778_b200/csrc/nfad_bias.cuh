@@ -85,14 +85,32 @@ __device__ __forceinline__ void bias_forward_packet(const uint4& rx, const float
     constexpr int V = S::kVec;
     float vx[V], vy[V], vd[V];
     S::unpack(rx, vx);
+    // the same width per call as the plain pass uses for this kind (two elements on packed fp32 arithmetic for the
+    // GELU-erf training forward and the value-only GELU forwards of 16-bit storage; the same bits either way)
+    constexpr bool kPairs = kTrain ? ForwardTrainOp<K, P>::kPairs : ForwardInferOp<K, P>::kPairs;
+    if constexpr (kPairs) {
 #pragma unroll
-    for (int e = 0; e < V; ++e) {
-        if (kTrain) {
-            ActOut o = evaluate<K, P>(bias_sum(vx[e], vb[e]));
-            vy[e] = o.y;
-            vd[e] = o.dydx;
-        } else {
-            vy[e] = evaluate_value(K{}, P{}, bias_sum(vx[e], vb[e]));
+        for (int e = 0; e < V; e += 2) {
+            const float2 z = make_float2(bias_sum(vx[e], vb[e]), bias_sum(vx[e + 1], vb[e + 1]));
+            if (kTrain) {
+                ActOut2 o = evaluate(K{}, Fast2{}, z);
+                vy[e] = o.y.x; vy[e + 1] = o.y.y;
+                vd[e] = o.dydx.x; vd[e + 1] = o.dydx.y;
+            } else {
+                float2 y2 = evaluate_value(K{}, Fast2{}, z);
+                vy[e] = y2.x; vy[e + 1] = y2.y;
+            }
+        }
+    } else {
+#pragma unroll
+        for (int e = 0; e < V; ++e) {
+            if (kTrain) {
+                ActOut o = evaluate<K, P>(bias_sum(vx[e], vb[e]));
+                vy[e] = o.y;
+                vd[e] = o.dydx;
+            } else {
+                vy[e] = evaluate_value(K{}, P{}, bias_sum(vx[e], vb[e]));
+            }
         }
     }
     store_packet<true>(y, S::pack(vy));
