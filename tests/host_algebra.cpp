@@ -97,3 +97,35 @@ extern "C" void host_algebra(int kind, int width, const float* x, float* y, floa
     case 3: run<Mish>(width, x, y, d, v, h, n); break;
     }
 }
+
+// one general-purpose primitive applied to the dual (x, 1): value and tangent.  op: 0 exp, 1 log1p, 2 tanh, 3 erf,
+// 4 softplus, 5 sigmoid, 6 (1 + tanh)/2, 7 (1 + erf)/2.  wide: 0 fp32 arithmetic, 1 double.
+template <class D, class T> static void prim(int op, T x, T* v, T* t)
+{
+    D a{x, T(1)}, r{T(0), T(0)};
+    switch (op) {
+    case 0: r = dual_exp(a); break;
+    case 1: r = dual_log1p(a); break;
+    case 2: r = dual_tanh(a); break;
+    case 3: r = dual_erf(a); break;
+    case 4: r = dual_softplus(a); break;
+    case 5: r = as_dual(dual_sigmoid(a)); break;
+    case 6: r = as_dual(dual_half_one_plus_tanh(a)); break;
+    case 7: r = as_dual(dual_half_one_plus_erf(a)); break;
+    }
+    *v = r.v;
+    *t = r.t;
+}
+extern "C" void host_primitive(int op, int wide, const double* x, double* v, double* t, size_t n)
+{
+    for (size_t i = 0; i < n; ++i) {
+        if (wide) {
+            prim<Dual<Wide>, double>(op, x[i], &v[i], &t[i]);
+        } else {
+            float fv, ft;
+            prim<Dual<Fast>, float>(op, (float)x[i], &fv, &ft);
+            v[i] = fv;
+            t[i] = ft;
+        }
+    }
+}

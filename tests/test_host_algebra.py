@@ -32,6 +32,8 @@ def host(tmp_path_factory):
     lib = ctypes.CDLL(so)
     lib.host_algebra.argtypes = [ctypes.c_int, ctypes.c_int] + [ctypes.c_void_p] * 5 + [ctypes.c_size_t]
     lib.host_algebra.restype = None
+    lib.host_primitive.argtypes = [ctypes.c_int, ctypes.c_int] + [ctypes.c_void_p] * 3 + [ctypes.c_size_t]
+    lib.host_primitive.restype = None
 
     def run(kind: str, width: int, x: np.ndarray):
         x = np.ascontiguousarray(x, np.float32)
@@ -39,6 +41,13 @@ def host(tmp_path_factory):
         lib.host_algebra(KINDS.index(kind), width, x.ctypes.data, *[o.ctypes.data for o in out], x.size)
         return out                                   # y, f', value-only y, gate
 
+    def primitive(op: int, wide: bool, x: np.ndarray):
+        x = np.ascontiguousarray(x, np.float64)
+        v, t = np.empty_like(x), np.empty_like(x)
+        lib.host_primitive(op, int(wide), x.ctypes.data, v.ctypes.data, t.ctypes.data, x.size)
+        return v, t
+
+    run.primitive = primitive
     return run
 
 
@@ -105,3 +114,48 @@ def test_non_finite_and_saturated_inputs(host, kind):
         assert y[2] == 0.0 and np.signbit(y[2]) and d[2] == 0.0
         assert abs(y[3] - 1000.0) <= 1000.0 * tol and abs(d[3] - 1.0) <= tol and abs(v[3] - 1000.0) <= 1000.0 * tol
         assert y[4] == 0.0 and d[4] == 0.0 and v[4] == 0.0
+
+
+def _reference_primitives():
+    """(name, value, derivative, domain) of each general-purpose primitive, from mpmath at 50 digits."""
+    mp = pytest.importorskip("mpmath")
+    mp.mp.dps = 50
+    sig = lambda a: 1 / (1 + mp.exp(-a))
+    return mp, [
+        ("exp", mp.exp, mp.exp, (-80.0, 80.0)),
+        ("log1p", mp.log1p, lambda a: 1 / (1 + a), (-0.99, 1.0e6)),
+        ("tanh", mp.tanh, lambda a: mp.sech(a) ** 2, (-12.0, 12.0)),
+        ("erf", mp.erf, lambda a: 2 / mp.sqrt(mp.pi) * mp.exp(-a * a), (-5.0, 5.0)),
+        ("softplus", lambda a: mp.log1p(mp.exp(a)), sig, (-80.0, 80.0)),
+        ("sigmoid", sig, lambda a: sig(a) * sig(-a), (-80.0, 80.0)),
+        ("(1+tanh)/2", lambda a: sig(2 * a), lambda a: 2 * sig(2 * a) * sig(-2 * a), (-40.0, 40.0)),
+        ("(1+erf)/2", lambda a: mp.erfc(-a) / 2, lambda a: mp.exp(-a * a) / mp.sqrt(mp.pi), (-9.0, 9.0)),
+    ]
+
+
+@pytest.mark.parametrize("wide", [False, True])
+def test_general_purpose_primitives(host, wide):
+    """Section III-A's primitive set as the sequences use it: value and tangent of each primitive at (x, 1) against
+    50-digit arithmetic, relative to the result (these points avoid the zero of tanh and erf, where the value itself
+    is tiny and the absolute error is what stays small).  fp32 arithmetic: 2^-18 with exact stand-ins for the
+    approximate units; double: 2^-40."""
+    mp, prims = _reference_primitives()
+    rng = np.random.default_rng(7)
+    tol = 2.0 ** -40 if wide else 2.0 ** -18
+    # fp32 arithmetic forms exp(a) from one rounding of a log2(e): its relative error grows like |a| 2^-24, so the
+    # fp32 primitives are compared where |a| is moderate
+    narrow = {"exp": 8.0, "tanh": 8.0, "erf": 3.0, "softplus": 8.0, "sigmoid": 8.0, "(1+tanh)/2": 4.0, "(1+erf)/2": 3.0}
+    for op, (name, f, df, (lo, hi)) in enumerate(prims):
+        if not wide:
+            lo, hi = (-narrow[name], narrow[name]) if name in narrow else (lo, 1.0e4)
+        x = rng.uniform(lo, hi, 400)
+        if not wide:
+            x = x.astype(np.float32).astype(np.float64)
+        x = x[np.abs(x) > 1e-3]
+        v, t = host.primitive(op, wide, x)
+        for xi, vi, ti in zip(x, v, t):
+            fv, ft = f(mp.mpf(float(xi))), df(mp.mpf(float(xi)))
+            # the fp32 erfc fit is built for 16-bit results: 2^-16 of erfc itself, i.e. 2^-15 with the operations around it
+            tl = 2.0 ** -15 if (not wide and "erf" in name) else tol
+            assert abs(mp.mpf(float(vi)) - fv) <= tl * abs(fv), (name, "value", xi, vi, float(fv))
+            assert abs(mp.mpf(float(ti)) - ft) <= tl * abs(ft), (name, "tangent", xi, ti, float(ft))
